@@ -1,0 +1,174 @@
+/*
+ * straggler_sim.h - C ABI of the batched simulator of distributed SGD with straggling workers
+ * (K-sync, K-batch-sync, K-async, K-batch-async SGD and a growing-K schedule), after
+ * "Slow and Stale Gradients Can Win the Race" (Dutta, Wang, Joshi; arXiv 2003.10579).
+ *
+ * One handle simulates n_replicas independent parameter servers, each with P workers, on the
+ * current CUDA device.  Everything runs in CUDA kernels for sm_100a; there is no CPU path.
+ *
+ * Conventions
+ *   - Every call returns a sim_status and never throws or aborts.  Outputs are defined only on
+ *     SIM_OK.  sim_last_error() gives a message for the last failure of a handle
+ *     (sim_last_error(NULL): of the last failed sim_create / handle-less call on this thread).
+ *   - "device" pointers are CUDA device pointers on the device that was current at sim_create;
+ *     "host" pointers are ordinary host memory.  The library never takes ownership of a
+ *     caller's buffer.  The data set (X, y / label, w_ref) is borrowed: it must stay valid and
+ *     unchanged until sim_destroy.  The library allocates only its own state and trace.
+ *   - Work is enqueued on the stream given at sim_create (a cudaStream_t passed as void*, NULL =
+ *     the legacy default stream).  sim_run returns after enqueueing; sim_get_* and
+ *     sim_trace_size synchronise that stream first and report a device-side error then.
+ *   - Random streams are counter-based (Philox4x32-10, key = seed) and keyed by (global replica
+ *     id, worker, the worker's task sequence number), so results do not depend on how replicas
+ *     are split over handles or GPUs: replica r of a handle has global id replica_base + r.
+ */
+#ifndef STRAGGLER_SIM_H
+#define STRAGGLER_SIM_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SIM_MAX_P 32          /* workers per replica (one warp lane each in the arrival kernels) */
+#define SIM_MAX_CLASSES 16    /* softmax / MLP outputs */
+
+typedef struct sim_handle sim_handle;   /* opaque; owned by the library */
+
+typedef enum {
+  SIM_OK = 0,
+  SIM_ERR_ARG = 1,       /* invalid argument, detected on the host before any launch */
+  SIM_ERR_ALLOC = 2,     /* device or host allocation failed */
+  SIM_ERR_CUDA = 3,      /* a CUDA runtime call or a kernel launch failed */
+  SIM_ERR_TIMEOUT = 4,   /* a bounded device-side wait ran out; the handle is unusable */
+  SIM_ERR_STATE = 5,     /* call not allowed in this state (e.g. sim_set_params after sim_run) */
+  SIM_ERR_INTERNAL = 6   /* an internal consistency check failed on the device */
+} sim_status;
+
+/* The four variants of Section 2.2 ("Variants of SGD"). */
+typedef enum {
+  SIM_KSYNC = 0,        /* wait for the first K of P workers, cancel the rest; Eq. 2 */
+  SIM_KBATCHSYNC = 1,   /* first K minibatches, finishers start another at the same w_j; Eq. 2 */
+  SIM_KASYNC = 2,       /* first K of P workers, others keep their stale parameters; Eq. 3 */
+  SIM_KBATCHASYNC = 3   /* every K pushes from anyone, pusher refetches at once; Eq. 3 */
+} sim_variant;
+
+/* The per-sample loss f(w, xi) of the empirical risk, Eq. 1. */
+typedef enum {
+  SIM_NONE = 0,      /* no parameters: arrival process and clock only (the runtime results of Section 3) */
+  SIM_LSQ = 1,       /* f = 1/2 (x.w - y)^2,                         n_params = d */
+  SIM_LOGISTIC = 2,  /* label b in {0,1}: f = softplus(x.w) - b x.w, n_params = d */
+  SIM_SOFTMAX = 3,   /* f = -log softmax(W x)[label], W [n_classes][d] row-major, n_params = n_classes*d */
+  SIM_MLP2 = 4       /* relu MLP d-hidden-n_classes with biases, cross-entropy; parameters
+                        [W1 (d x hidden row-major), b1, W2 (hidden x n_classes), b2]; the two products
+                        over d take bf16 operands (x, W1, delta1) with fp32 accumulation */
+} sim_model;
+
+/* Per-minibatch compute time X of a worker, i.i.d. over workers and minibatches (Section 3.1):
+ * X = Exp(mu) (rate mu, mean 1/mu) or shift + Exp(mu) (Lemma 4's shifted exponential). */
+typedef enum { SIM_DELAY_EXP = 0, SIM_DELAY_SHIFTED_EXP = 1 } sim_delay_kind;
+typedef struct { sim_delay_kind kind; double mu; double shift; } sim_delay;
+
+/* The data set S of N samples (Section 2).  All pointers are DEVICE pointers, borrowed. */
+typedef struct {
+  sim_model model;
+  int64_t n;             /* samples, 1 <= n <= 2^32 */
+  int32_t d;             /* features per sample, d % 4 == 0 */
+  int32_t n_classes;     /* SOFTMAX / MLP2: 2..SIM_MAX_CLASSES; otherwise ignored */
+  int32_t hidden;        /* MLP2: hidden width; otherwise ignored */
+  const float* X;        /* [n][d] row-major fp32, 16-byte aligned */
+  const float* y;        /* LSQ: [n] fp32 targets; otherwise NULL */
+  const int32_t* label;  /* LOGISTIC: [n] in {0,1}; SOFTMAX / MLP2: [n] in [0, n_classes); LSQ: NULL */
+  const float* w_ref;    /* optional [n_params]: |w_{j+1} - w_ref|^2 is recorded per update; may be NULL */
+} sim_problem;
+
+/*
+ * Create a simulation: P workers, K of them (or K minibatches) per update, step size eta
+ * (Eq. 2 / Eq. 3: w_{j+1} = w_j - (eta/K) sum_l g(w_tau(l,j), xi_l,j)), minibatch size m per
+ * worker, drawn with replacement from all n samples.  Initial parameters are zero until
+ * sim_set_params.  problem may be NULL or have model SIM_NONE for a clock-only simulation.
+ * Errors: SIM_ERR_ARG for P not in [1, SIM_MAX_P], K not in [1, P], m < 1, n_replicas < 1,
+ * mu <= 0 or NaN, shift < 0 or not finite, d % 4 != 0, misaligned or NULL X, missing y / label,
+ * replica ids beyond 2^32; SIM_ERR_ALLOC / SIM_ERR_CUDA otherwise.  *out is NULL on failure.
+ */
+sim_status sim_create(const sim_problem* problem, int32_t P, int32_t K, sim_variant variant,
+                      sim_delay delay, float eta, int32_t m, uint64_t seed, int32_t n_replicas,
+                      int64_t replica_base, void* cuda_stream, sim_handle** out);
+
+/* Same w0 (DEVICE, [n_params]) for every replica.  Only before the first sim_run (SIM_ERR_STATE
+ * after).  The buffer is read during the call's enqueued work, not kept. */
+sim_status sim_set_params(sim_handle* h, const float* w0);
+
+/* Growing-K schedule with the interval structure of Algorithm 1 (Section 6): an update that
+ * starts at simulated time t uses K = min(P, K0 * 2^floor(t / t_interval)).  t_interval <= 0
+ * switches it off (fixed K from sim_create).  Only before the first sim_run. */
+sim_status sim_set_adasync(sim_handle* h, int32_t K0, double t_interval);
+
+/* Optional performance knob: depth of the shared-memory ring that stages sample rows ahead of
+ * the arithmetic (2..8; 0 = chosen from d).  Results do not depend on it. */
+sim_status sim_set_tuning(sim_handle* h, int32_t stages);
+
+/* Optional: make room for total_updates updates of trace now, so that later sim_run calls
+ * allocate nothing. */
+sim_status sim_reserve(sim_handle* h, int64_t total_updates);
+
+/* Advance every replica by `iters` server updates.  Resumable: run(a); run(b) gives the same
+ * bits as run(a+b).  Enqueues on the handle's stream and returns. */
+sim_status sim_run(sim_handle* h, int64_t iters);
+
+/* Updates done so far and the row length K_max of the per-contributor trace arrays
+ * (K, or P when the growing-K schedule is on). */
+sim_status sim_trace_size(const sim_handle* h, int64_t* n_updates, int32_t* K_max);
+
+/*
+ * Copy the trace of all J = n_updates updates of all R = n_replicas replicas into caller-owned
+ * DEVICE buffers; any pointer may be NULL to skip that array.  Section 2.3's two metrics are
+ * error and wall-clock runtime: t is the simulated clock at update j, loss the minibatch loss
+ * (1/(K m)) sum_l sum_q f(w_tau(l,j); xi) of the gradients used, dist2 = |w_{j+1} - w_ref|^2
+ * (0 without w_ref).  worker / stale / seq list the K_used[j] contributors in arrival order
+ * (staleness j - tau(l,j) of Eq. 3; seq = that worker's task sequence number), padded with
+ * 0xFFFF / 0xFFFFFFFF up to K_max.  loss and dist2 are 0 for SIM_NONE.
+ */
+sim_status sim_get_trace(const sim_handle* h, double* t /*[R][J]*/, float* loss /*[R][J]*/,
+                         float* dist2 /*[R][J]*/, uint16_t* K_used /*[R][J]*/,
+                         uint16_t* worker /*[R][J][K_max]*/, uint32_t* stale /*[R][J][K_max]*/,
+                         uint32_t* seq /*[R][J][K_max]*/);
+
+/* Current parameters w_j of every replica into a DEVICE buffer [R][n_params]. */
+sim_status sim_get_params(const sim_handle* h, float* w);
+
+/* Number of parameters of the handle's model (0 for SIM_NONE). */
+int64_t sim_n_params(const sim_handle* h);
+
+const char* sim_last_error(const sim_handle* h);
+void sim_destroy(sim_handle* h);
+
+/*
+ * The random draws on their own (Section 3.1's X_i and Section 2's minibatches), for checking a
+ * stream against another implementation.  DEVICE outputs, enqueued on `cuda_stream`:
+ *   sim_draw_delays:  out[(r*P + i)*n_seq + s] = compute time of task s of worker i of global
+ *                     replica replica_base + r
+ *   sim_draw_indices: out[((r*P + i)*n_seq + s)*m + q] = sample index q of that task's minibatch
+ */
+sim_status sim_draw_delays(sim_delay delay, uint64_t seed, int64_t replica_base, int32_t n_replicas,
+                           int32_t P, int32_t n_seq, double* out, void* cuda_stream);
+sim_status sim_draw_indices(uint64_t seed, int64_t replica_base, int32_t n_replicas, int32_t P,
+                            int32_t n_seq, int64_t n, int32_t m, uint32_t* out, void* cuda_stream);
+
+/*
+ * One-shot call on HOST buffers: copies the data set to the device, creates a simulation,
+ * runs `iters` updates, copies the trace (same arrays and layout as sim_get_trace, any may be
+ * NULL) and the final parameters ([R][n_params], may be NULL) back to host memory, and frees
+ * everything.  `problem` holds HOST pointers here.  w0 (host, [n_params]) may be NULL for zeros;
+ * K0 / t_interval as in sim_set_adasync.
+ */
+sim_status sim_simulate_host(const sim_problem* problem, int32_t P, int32_t K, sim_variant variant,
+                             sim_delay delay, float eta, int32_t m, uint64_t seed, int32_t n_replicas,
+                             int64_t replica_base, const float* w0, int32_t K0, double t_interval,
+                             int64_t iters, double* t, float* loss, float* dist2, uint16_t* K_used,
+                             uint16_t* worker, uint32_t* stale, uint32_t* seq, float* w_final);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* STRAGGLER_SIM_H */

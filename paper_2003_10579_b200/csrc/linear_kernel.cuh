@@ -1,0 +1,391 @@
+// Gradient / update kernel for the single-output linear models (least squares, logistic).
+//
+// One CTA per replica walks the replica's schedule: for each update j, for each contributor l
+// in arrival order, the m rows of its minibatch (indices re-derived from the Philox stream) are
+// staged into shared memory by bulk asynchronous copies (one 4d-byte copy per row, completion
+// counted on an mbarrier), several tiles ahead of the arithmetic - the rows never depend on w,
+// so the row stream can be prefetched across contributor and update boundaries.  Per tile of T
+// rows:   z_q = x_q . w_tau        (each thread owns a fixed set of columns; block reduction)
+//         a_q = dl/dz(z_q, y_q)    (x.w - y, or sigmoid(x.w) - b)
+//         g  += sum_q a_q x_q      (column owner accumulates, no reduction needed)
+// and at the end of the update  w_{j+1} = w_j - (eta / (K m)) g   (Eq. 2 / Eq. 3), the minibatch
+// loss and |w_{j+1} - w_ref|^2 are recorded.  w_j, w_tau and g live in registers; for the
+// asynchronous variants every version is also written to the replica's version pool, from
+// which stale snapshots w_tau are read back.
+#pragma once
+#include "schedule_kernel.cuh"
+
+namespace ssim {
+
+enum : int { M_NONE = 0, M_LSQ = 1, M_LOGISTIC = 2, M_SOFTMAX = 3, M_MLP2 = 4 };
+
+struct NumericArgs {
+  const float* X;            // [n][d]
+  const void* y;             // [n] float targets (lsq) or int32 labels
+  const float* w_ref;        // [n_params] or null
+  uint64_t n;
+  int d, m, model, n_classes;
+  float eta;
+  uint64_t seed;
+  uint32_t replica_base;
+  int R;
+  long long j0, iters, cap;
+  int K_stride;
+  int is_async;
+  int n_slots;
+  long long n_params;
+  const uint16_t* K_used;    // schedule, see schedule_kernel.cuh
+  const uint16_t* worker;
+  const uint32_t* seq;
+  const uint8_t* snap_slot;
+  const uint8_t* new_slot;
+  const uint8_t* begin_slot; // [R] slot of w_{j0}
+  float* loss;               // [R][cap]
+  float* dist2;              // [R][cap]
+  float* w_state;            // synchronous variants: [R][n_params]
+  float* pool;               // asynchronous variants: [R][n_slots][n_params]
+  int stages;                // shared-memory ring depth
+  int* err;
+};
+
+// ---- shared-memory barrier and bulk-copy primitives ------------------------------------------
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_fence_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: gives up after a few seconds' worth of polls and reports it.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < (1u << 24); ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (i > 4096) __nanosleep(128);
+  }
+  return false;
+}
+// global -> shared bulk copy of `bytes` (multiple of 16, both addresses 16-byte aligned)
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+      ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// 4-byte asynchronous copy whose completion is counted as one arrival on `bar`
+__device__ __forceinline__ void word_g2s_arrive(uint32_t dst, const void* src, uint32_t bar) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
+  return v;
+}
+
+// ---- the producer's walk over the schedule ---------------------------------------------------
+enum : int { TILE_FIRST_OF_TASK = 1, TILE_LAST_OF_TASK = 2, TILE_LAST_OF_UPDATE = 4, TILE_LAST_OF_RUN = 8 };
+
+struct TileInfo { int flags, rows, K, snap, fresh; };   // 5 ints per stage in shared memory
+
+struct TaskDesc { uint32_t worker, seq, snap, fresh, K; };
+
+struct ScheduleWalk {
+  long long j, j_end, row0;   // current update, end of run, r * cap
+  int l, k, tiles_per_task;
+  TaskDesc cur, nxt;
+  bool done;
+
+  __device__ __forceinline__ TaskDesc load(const NumericArgs& a, long long jj, int ll) const {
+    TaskDesc t;
+    const long long row = row0 + jj;
+    t.worker = a.worker[row * a.K_stride + ll];
+    t.seq = a.seq[row * a.K_stride + ll];
+    t.K = a.K_used[row];
+    t.snap = a.is_async ? a.snap_slot[row * a.K_stride + ll] : 0u;
+    t.fresh = a.is_async ? a.new_slot[row] : 0u;
+    return t;
+  }
+  __device__ __forceinline__ void prefetch_next(const NumericArgs& a) {
+    long long nj = j; int nl = l + 1;
+    if (nl >= (int)cur.K) { nl = 0; nj = j + 1; }
+    if (nj < j_end) nxt = load(a, nj, nl);
+  }
+  __device__ __forceinline__ void start(const NumericArgs& a, int r) {
+    row0 = (long long)r * a.cap; j = a.j0; j_end = a.j0 + a.iters; l = 0; k = 0;
+    tiles_per_task = (a.m + 0) ;   // set by caller (depends on T)
+    done = a.iters <= 0;
+    if (!done) { cur = load(a, j, 0); prefetch_next(a); }
+  }
+  __device__ __forceinline__ void advance(const NumericArgs& a) {
+    if (++k < tiles_per_task) return;
+    k = 0;
+    if (++l >= (int)cur.K) { l = 0; ++j; }
+    if (j >= j_end) { done = true; return; }
+    cur = nxt;
+    prefetch_next(a);
+  }
+};
+
+template <int NT, int CHUNKS, int T, bool ASYNC>
+__global__ void __launch_bounds__(NT) linear1_kernel(NumericArgs a) {
+  constexpr int NW = NT / 32;
+  constexpr int E = 4 * CHUNKS;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int r = blockIdx.x;
+  const int d = a.d, d4 = d >> 2, S = a.stages, m = a.m;
+  const uint32_t rid = a.replica_base + (uint32_t)r;
+  const uint32_t row_bytes = (uint32_t)d * 4u;
+
+  extern __shared__ __align__(128) unsigned char smem[];
+  // layout: [S] barriers | [S] TileInfo | y_stage [S][T] | red [2][NW][T] | misc [NW] | rows [S][T][d]
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem);
+  TileInfo* info_s = reinterpret_cast<TileInfo*>(smem + 8 * S);
+  uint32_t* y_s = reinterpret_cast<uint32_t*>(info_s + S);
+  float* red_s = reinterpret_cast<float*>(y_s + S * T);
+  float* misc_s = red_s + 2 * NW * T;
+  const size_t head = (size_t)((unsigned char*)(misc_s + NW) - smem);
+  float* rows_s = reinterpret_cast<float*>(smem + ((head + 127) & ~(size_t)127));
+
+  if (tid == 0) {
+    for (int s = 0; s < S; ++s) mbar_init(smem_addr(&full[s]), (uint32_t)T + 1u);
+    mbar_fence_init();
+  }
+  __syncthreads();
+
+  // ---- parameters in registers: thread owns float4 chunks tid + NT*c ----
+  float w_cur[E], w_tau[E], g[E];
+  int cur_slot = ASYNC ? (int)a.begin_slot[r] : 0;
+  {
+    const float* src = ASYNC ? a.pool + ((size_t)r * a.n_slots + cur_slot) * (size_t)d
+                             : a.w_state + (size_t)r * d;
+#pragma unroll
+    for (int c = 0; c < CHUNKS; ++c) {
+      const int ci = tid + NT * c;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (ci < d4) v = reinterpret_cast<const float4*>(src)[ci];
+      w_cur[4 * c] = v.x; w_cur[4 * c + 1] = v.y; w_cur[4 * c + 2] = v.z; w_cur[4 * c + 3] = v.w;
+    }
+#pragma unroll
+    for (int e = 0; e < E; ++e) { g[e] = 0.f; w_tau[e] = w_cur[e]; }
+  }
+
+  // ---- producer (warp 0): stage tiles of rows ahead of the arithmetic ----
+  ScheduleWalk walk;
+  walk.done = true;
+  auto issue_tile = [&](long long tile_no) {
+    // called by all lanes of warp 0; the stage's previous contents have been consumed
+    if (walk.done) return;
+    const int st = (int)(tile_no % S);
+    const uint32_t bar = smem_addr(&full[st]);
+    const int rows = min(T, m - walk.k * T);
+    if (lane == 0) {
+      TileInfo ti;
+      ti.rows = rows; ti.K = (int)walk.cur.K; ti.snap = (int)walk.cur.snap; ti.fresh = (int)walk.cur.fresh;
+      ti.flags = (walk.k == 0 ? TILE_FIRST_OF_TASK : 0) | (walk.k == walk.tiles_per_task - 1 ? TILE_LAST_OF_TASK : 0);
+      if ((ti.flags & TILE_LAST_OF_TASK) && walk.l == (int)walk.cur.K - 1) {
+        ti.flags |= TILE_LAST_OF_UPDATE;
+        if (walk.j == walk.j_end - 1) ti.flags |= TILE_LAST_OF_RUN;
+      }
+      info_s[st] = ti;
+      mbar_arrive_expect_tx(bar, (uint32_t)rows * row_bytes);
+    }
+    __syncwarp();
+    if (lane < T) {
+      if (lane < rows) {
+        const uint32_t q = (uint32_t)(walk.k * T + lane);
+        uint32_t idx = draw_index(a.seed, rid, walk.cur.worker, walk.cur.seq, q, a.n);
+        if ((uint64_t)idx >= a.n) { atomicExch(a.err, ERR_BAD_INDEX); idx = 0; }
+        bulk_g2s(smem_addr(rows_s + ((size_t)st * T + lane) * d), a.X + (size_t)idx * d, row_bytes, bar);
+        word_g2s_arrive(smem_addr(&y_s[st * T + lane]), reinterpret_cast<const uint32_t*>(a.y) + idx, bar);
+      } else {
+        mbar_arrive(bar);
+      }
+    }
+    walk.advance(a);
+  };
+  if (warp == 0) {
+    walk.start(a, r);
+    walk.tiles_per_task = (m + T - 1) / T;
+    for (int s = 0; s < S - 1; ++s) issue_tile(s);
+  }
+  __syncthreads();
+  if (a.iters <= 0) return;
+
+  float loss_acc = 0.f;
+  long long j = a.j0;
+  bool failed = false;
+  for (long long it = 0;; ++it) {
+    const int st = (int)(it % S);
+    const uint32_t parity = (uint32_t)((it / S) & 1);
+    if (!mbar_wait(smem_addr(&full[st]), parity)) { failed = true; break; }
+    const TileInfo ti = info_s[st];
+    const float* tile = rows_s + (size_t)st * T * d;
+
+    if (ASYNC && (ti.flags & TILE_FIRST_OF_TASK)) {
+      if (ti.snap == cur_slot) {
+#pragma unroll
+        for (int e = 0; e < E; ++e) w_tau[e] = w_cur[e];
+      } else {
+        const float4* src = reinterpret_cast<const float4*>(a.pool + ((size_t)r * a.n_slots + ti.snap) * (size_t)d);
+#pragma unroll
+        for (int c = 0; c < CHUNKS; ++c) {
+          const int ci = tid + NT * c;
+          float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (ci < d4) v = src[ci];
+          w_tau[4 * c] = v.x; w_tau[4 * c + 1] = v.y; w_tau[4 * c + 2] = v.z; w_tau[4 * c + 3] = v.w;
+        }
+      }
+    }
+
+    // ---- z_q = x_q . w_tau: per-thread partial over own columns, then block reduction ----
+    float part[T];
+#pragma unroll
+    for (int q = 0; q < T; ++q) part[q] = 0.f;
+#pragma unroll
+    for (int c = 0; c < CHUNKS; ++c) {
+      const int ci = tid + NT * c;
+      if (ci < d4) {
+#pragma unroll
+        for (int q = 0; q < T; ++q) {
+          if (q < ti.rows) {
+            const float4 x = reinterpret_cast<const float4*>(tile + (size_t)q * d)[ci];
+            const float* wt = ASYNC ? &w_tau[4 * c] : &w_cur[4 * c];
+            part[q] = fmaf(x.x, wt[0], part[q]);
+            part[q] = fmaf(x.y, wt[1], part[q]);
+            part[q] = fmaf(x.z, wt[2], part[q]);
+            part[q] = fmaf(x.w, wt[3], part[q]);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int q = 0; q < T; ++q) part[q] = warp_sum(part[q]);
+    if (lane == 0) {
+#pragma unroll
+      for (int q = 0; q < T; ++q) red_s[((it & 1) * NW + warp) * T + q] = part[q];
+    }
+    __syncthreads();
+    // every thread is past its reads of the previous tile's stage: refill it
+    if (warp == 0) issue_tile(it + S - 1);
+
+    // ---- a_q = dl/dz and the loss ----
+    float aq[T];
+#pragma unroll
+    for (int q = 0; q < T; ++q) {
+      aq[q] = 0.f;
+      if (q < ti.rows) {
+        float z = 0.f;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) z += red_s[((it & 1) * NW + w) * T + q];
+        const uint32_t yraw = y_s[st * T + q];
+        if (a.model == M_LSQ) {
+          const float res = z - __uint_as_float(yraw);
+          aq[q] = res;
+          loss_acc = fmaf(0.5f * res, res, loss_acc);
+        } else {  // logistic, label b in {0,1}: f = softplus(z) - b z, df/dz = sigmoid(z) - b
+          const float b = (float)(int)yraw;
+          const float ez = expf(-fabsf(z));
+          const float sig = z >= 0.f ? 1.f / (1.f + ez) : ez / (1.f + ez);
+          aq[q] = sig - b;
+          loss_acc += fmaxf(z, 0.f) + log1pf(ez) - b * z;
+        }
+      }
+    }
+    // ---- g += sum_q a_q x_q over own columns ----
+#pragma unroll
+    for (int c = 0; c < CHUNKS; ++c) {
+      const int ci = tid + NT * c;
+      if (ci < d4) {
+#pragma unroll
+        for (int q = 0; q < T; ++q) {
+          if (q < ti.rows) {
+            const float4 x = reinterpret_cast<const float4*>(tile + (size_t)q * d)[ci];
+            g[4 * c] = fmaf(aq[q], x.x, g[4 * c]);
+            g[4 * c + 1] = fmaf(aq[q], x.y, g[4 * c + 1]);
+            g[4 * c + 2] = fmaf(aq[q], x.z, g[4 * c + 2]);
+            g[4 * c + 3] = fmaf(aq[q], x.w, g[4 * c + 3]);
+          }
+        }
+      }
+    }
+
+    if (ti.flags & TILE_LAST_OF_UPDATE) {
+      // w_{j+1} = w_j - (eta / (K m)) sum of the K m per-sample gradients
+      const float scale = (float)((double)a.eta / ((double)ti.K * (double)m));
+      float dd = 0.f;
+#pragma unroll
+      for (int c = 0; c < CHUNKS; ++c) {
+        const int ci = tid + NT * c;
+        if (ci < d4) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) { w_cur[4 * c + e] = fmaf(-scale, g[4 * c + e], w_cur[4 * c + e]); g[4 * c + e] = 0.f; }
+          if (ASYNC) {
+            float4* dst = reinterpret_cast<float4*>(a.pool + ((size_t)r * a.n_slots + ti.fresh) * (size_t)d);
+            dst[ci] = make_float4(w_cur[4 * c], w_cur[4 * c + 1], w_cur[4 * c + 2], w_cur[4 * c + 3]);
+          }
+          if (a.w_ref) {
+            const float4 wr = reinterpret_cast<const float4*>(a.w_ref)[ci];
+            const float e0 = w_cur[4 * c] - wr.x, e1 = w_cur[4 * c + 1] - wr.y, e2 = w_cur[4 * c + 2] - wr.z, e3 = w_cur[4 * c + 3] - wr.w;
+            dd = fmaf(e0, e0, dd); dd = fmaf(e1, e1, dd); dd = fmaf(e2, e2, dd); dd = fmaf(e3, e3, dd);
+          }
+        }
+      }
+      if (ASYNC) cur_slot = ti.fresh;
+      if (a.w_ref) {
+        dd = warp_sum(dd);
+        if (lane == 0) misc_s[warp] = dd;
+        __syncthreads();
+        if (tid == 0) {
+          float tot = 0.f;
+          for (int w = 0; w < NW; ++w) tot += misc_s[w];
+          a.dist2[(size_t)r * a.cap + j] = tot;
+        }
+      } else if (tid == 0) {
+        a.dist2[(size_t)r * a.cap + j] = 0.f;
+      }
+      if (tid == 0) a.loss[(size_t)r * a.cap + j] = loss_acc / ((float)ti.K * (float)m);
+      loss_acc = 0.f;
+      ++j;
+    }
+    if (ti.flags & TILE_LAST_OF_RUN) break;
+  }
+
+  if (failed) {
+    if (tid == 0) atomicExch(a.err, ERR_WAIT_TIMEOUT);
+    return;
+  }
+  if (!ASYNC) {
+    float4* dst = reinterpret_cast<float4*>(a.w_state + (size_t)r * d);
+#pragma unroll
+    for (int c = 0; c < CHUNKS; ++c) {
+      const int ci = tid + NT * c;
+      if (ci < d4) dst[ci] = make_float4(w_cur[4 * c], w_cur[4 * c + 1], w_cur[4 * c + 2], w_cur[4 * c + 3]);
+    }
+  }
+}
+
+// shared-memory bytes of linear1_kernel for a given shape
+inline size_t linear1_smem_bytes(int NT, int T, int S, int d) {
+  size_t head = 8 * (size_t)S + sizeof(TileInfo) * (size_t)S + 4 * (size_t)S * T + 4 * (size_t)2 * (NT / 32) * T + 4 * (size_t)(NT / 32);
+  head = (head + 127) & ~(size_t)127;
+  return head + (size_t)S * T * d * 4;
+}
+
+}  // namespace ssim

@@ -1,0 +1,548 @@
+// C-ABI of the straggler-SGD simulator: handle, argument checks, memory, kernel dispatch.
+// See include/straggler_sim.h for the contract of every entry point.
+#include "../../include/straggler_sim.h"
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "linear_kernel.cuh"
+#include "softmax_kernel.cuh"
+#include "mlp_kernel.cuh"
+
+using namespace ssim;
+
+namespace {
+
+thread_local std::string g_last_error;
+
+struct TraceBuffers {
+  double* t = nullptr;
+  float* loss = nullptr;
+  float* dist2 = nullptr;
+  uint16_t* K_used = nullptr;
+  uint16_t* worker = nullptr;
+  uint32_t* stale = nullptr;
+  uint32_t* seq = nullptr;
+  uint8_t* snap_slot = nullptr;
+  uint8_t* new_slot = nullptr;
+};
+
+}  // namespace
+
+struct sim_handle {
+  sim_problem prob{};
+  int P = 0, K = 0, variant = 0, m = 0, R = 0;
+  sim_delay delay{};
+  float eta = 0.f;
+  uint64_t seed = 0;
+  uint32_t replica_base = 0;
+  cudaStream_t stream = nullptr;
+  int device = 0;
+  int K0 = 0;
+  double t_interval = 0.0;
+  int K_stride = 0;
+  bool is_async = false;
+  int n_slots = 0;
+  long long n_params = 0;
+  long long n_updates = 0, cap = 0;
+  int tune_stages = 0;
+  // device state
+  uint32_t* s = nullptr;
+  uint32_t* tau = nullptr;
+  double* f = nullptr;
+  uint8_t* wslot = nullptr;
+  uint8_t* cur_slot = nullptr;
+  uint8_t* begin_slot = nullptr;
+  double* clock = nullptr;
+  float* w_state = nullptr;   // synchronous: [R][n_params]
+  float* pool = nullptr;      // asynchronous: [R][n_slots][n_params]
+  MlpScratch mlp{};
+  int* err = nullptr;
+  TraceBuffers tr;
+  bool poisoned = false;
+  mutable std::string last_error;
+};
+
+namespace {
+
+sim_status fail(const sim_handle* h, sim_status st, const std::string& msg) {
+  if (h) h->last_error = msg; else g_last_error = msg;
+  return st;
+}
+
+#define CUDA_TRY(h, expr)                                                                   \
+  do {                                                                                      \
+    cudaError_t e_ = (expr);                                                                \
+    if (e_ != cudaSuccess)                                                                  \
+      return fail(h, e_ == cudaErrorMemoryAllocation ? SIM_ERR_ALLOC : SIM_ERR_CUDA,       \
+                  std::string(#expr) + ": " + cudaGetErrorString(e_));                      \
+  } while (0)
+
+template <typename T>
+cudaError_t dev_alloc(T** p, size_t count, cudaStream_t st, bool zero = true) {
+  *p = nullptr;
+  if (count == 0) return cudaSuccess;
+  cudaError_t e = cudaMalloc(reinterpret_cast<void**>(p), count * sizeof(T));
+  if (e != cudaSuccess) { *p = nullptr; return e; }
+  if (zero) e = cudaMemsetAsync(*p, 0, count * sizeof(T), st);
+  return e;
+}
+
+long long model_params(const sim_problem& p) {
+  switch (p.model) {
+    case SIM_LSQ: case SIM_LOGISTIC: return p.d;
+    case SIM_SOFTMAX: return (long long)p.n_classes * p.d;
+    case SIM_MLP2: return (long long)p.d * p.hidden + p.hidden + (long long)p.hidden * p.n_classes + p.n_classes;
+    default: return 0;
+  }
+}
+
+sim_status check_delay(const sim_handle* h, const sim_delay& dl) {
+  if (dl.kind != SIM_DELAY_EXP && dl.kind != SIM_DELAY_SHIFTED_EXP) return fail(h, SIM_ERR_ARG, "unknown delay kind");
+  if (!(dl.mu > 0.0)) return fail(h, SIM_ERR_ARG, "delay rate mu must be > 0");
+  if (dl.kind == SIM_DELAY_SHIFTED_EXP && !(dl.shift >= 0.0 && std::isfinite(dl.shift)))
+    return fail(h, SIM_ERR_ARG, "delay shift must be finite and >= 0");
+  return SIM_OK;
+}
+
+__global__ void broadcast_params_kernel(const float* w0, float* dst, long long n_params, long long stride, int R) {
+  const long long total = n_params * R;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const long long r = i / n_params, p = i % n_params;
+    dst[r * stride + p] = w0[p];
+  }
+}
+
+__global__ void gather_params_kernel(const float* pool, const uint8_t* cur_slot, float* out, long long n_params, int n_slots, int R) {
+  const long long total = n_params * R;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const long long r = i / n_params, p = i % n_params;
+    out[i] = pool[(r * n_slots + cur_slot[r]) * n_params + p];
+  }
+}
+
+template <typename T>
+sim_status regrow(sim_handle* h, T** buf, size_t per_update, long long new_cap, bool zero) {
+  T* nb = nullptr;
+  CUDA_TRY(h, dev_alloc(&nb, (size_t)h->R * new_cap * per_update, h->stream, zero));
+  if (*buf && h->n_updates > 0) {
+    CUDA_TRY(h, cudaMemcpy2DAsync(nb, (size_t)new_cap * per_update * sizeof(T), *buf,
+                                  (size_t)h->cap * per_update * sizeof(T),
+                                  (size_t)h->n_updates * per_update * sizeof(T), h->R,
+                                  cudaMemcpyDeviceToDevice, h->stream));
+  }
+  if (*buf) { CUDA_TRY(h, cudaStreamSynchronize(h->stream)); cudaFree(*buf); }
+  *buf = nb;
+  return SIM_OK;
+}
+
+sim_status ensure_capacity(sim_handle* h, long long need) {
+  if (need <= h->cap) return SIM_OK;
+  long long nc = h->cap * 2 > need ? h->cap * 2 : need;
+  const size_t Ks = (size_t)h->K_stride;
+  sim_status st;
+  if ((st = regrow(h, &h->tr.t, 1, nc, false)) != SIM_OK) return st;
+  if ((st = regrow(h, &h->tr.loss, 1, nc, true)) != SIM_OK) return st;
+  if ((st = regrow(h, &h->tr.dist2, 1, nc, true)) != SIM_OK) return st;
+  if ((st = regrow(h, &h->tr.K_used, 1, nc, false)) != SIM_OK) return st;
+  if ((st = regrow(h, &h->tr.worker, Ks, nc, false)) != SIM_OK) return st;
+  if ((st = regrow(h, &h->tr.stale, Ks, nc, false)) != SIM_OK) return st;
+  if ((st = regrow(h, &h->tr.seq, Ks, nc, false)) != SIM_OK) return st;
+  if (h->is_async) {
+    if ((st = regrow(h, &h->tr.snap_slot, Ks, nc, false)) != SIM_OK) return st;
+    if ((st = regrow(h, &h->tr.new_slot, 1, nc, false)) != SIM_OK) return st;
+  }
+  h->cap = nc;
+  return SIM_OK;
+}
+
+// ---- dispatch of the single-output linear kernel by feature count ----
+template <int NT, int CHUNKS, int T>
+sim_status launch_linear1(sim_handle* h, NumericArgs& a) {
+  const int d = a.d;
+  const size_t row_bytes = (size_t)d * 4;
+  int S = h->tune_stages;
+  if (S <= 0) {
+    const size_t budget = d <= 1024 ? (36u << 10) : (200u << 10);
+    S = (int)(budget / ((size_t)T * row_bytes));
+  }
+  if (S < 2) S = 2;
+  if (S > 8) S = 8;
+  size_t smem = linear1_smem_bytes(NT, T, S, d);
+  while (smem > (size_t)(226 << 10) && S > 2) { --S; smem = linear1_smem_bytes(NT, T, S, d); }
+  if (smem > (size_t)(226 << 10)) return fail(h, SIM_ERR_ARG, "d too large for the row staging buffers");
+  a.stages = S;
+  auto kern = a.is_async ? linear1_kernel<NT, CHUNKS, T, true> : linear1_kernel<NT, CHUNKS, T, false>;
+  CUDA_TRY(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  kern<<<a.R, NT, smem, h->stream>>>(a);
+  CUDA_TRY(h, cudaGetLastError());
+  return SIM_OK;
+}
+
+sim_status run_linear1(sim_handle* h, NumericArgs& a) {
+  const int d4 = a.d / 4;
+  if (d4 <= 32) return launch_linear1<32, 1, 8>(h, a);
+  if (d4 <= 64) return launch_linear1<64, 1, 8>(h, a);
+  if (d4 <= 128) return launch_linear1<128, 1, 4>(h, a);
+  if (d4 <= 256) return launch_linear1<128, 2, 4>(h, a);
+  if (d4 <= 512) return launch_linear1<256, 2, 4>(h, a);
+  if (d4 <= 1024) return launch_linear1<256, 4, 4>(h, a);
+  if (d4 <= 2048) return launch_linear1<512, 4, 2>(h, a);
+  return fail(h, SIM_ERR_ARG, "d > 8192 is not supported by the linear-model kernel");
+}
+
+sim_status device_error(const sim_handle* h) {
+  int e = 0;
+  CUDA_TRY(h, cudaStreamSynchronize(h->stream));
+  CUDA_TRY(h, cudaMemcpy(&e, h->err, sizeof(int), cudaMemcpyDeviceToHost));
+  if (e == ERR_NONE) return SIM_OK;
+  const_cast<sim_handle*>(h)->poisoned = true;
+  if (e == ERR_WAIT_TIMEOUT) return fail(h, SIM_ERR_TIMEOUT, "a bounded device-side wait ran out");
+  return fail(h, SIM_ERR_INTERNAL, "device-side consistency check failed (code " + std::to_string(e) + ")");
+}
+
+void free_all(sim_handle* h) {
+  cudaFree(h->s); cudaFree(h->tau); cudaFree(h->f); cudaFree(h->wslot); cudaFree(h->cur_slot);
+  cudaFree(h->begin_slot); cudaFree(h->clock); cudaFree(h->w_state); cudaFree(h->pool); cudaFree(h->err);
+  mlp_scratch_free(h->mlp);
+  cudaFree(h->tr.t); cudaFree(h->tr.loss); cudaFree(h->tr.dist2); cudaFree(h->tr.K_used);
+  cudaFree(h->tr.worker); cudaFree(h->tr.stale); cudaFree(h->tr.seq); cudaFree(h->tr.snap_slot);
+  cudaFree(h->tr.new_slot);
+}
+
+}  // namespace
+
+extern "C" {
+
+sim_status sim_create(const sim_problem* problem, int32_t P, int32_t K, sim_variant variant,
+                      sim_delay delay, float eta, int32_t m, uint64_t seed, int32_t n_replicas,
+                      int64_t replica_base, void* cuda_stream, sim_handle** out) {
+  if (!out) return fail(nullptr, SIM_ERR_ARG, "out is NULL");
+  *out = nullptr;
+  if (P < 1 || P > SIM_MAX_P) return fail(nullptr, SIM_ERR_ARG, "P must be in [1, SIM_MAX_P]");
+  if (K < 1 || K > P) return fail(nullptr, SIM_ERR_ARG, "K must be in [1, P]");
+  if ((int)variant < 0 || (int)variant > 3) return fail(nullptr, SIM_ERR_ARG, "unknown variant");
+  if (m < 1) return fail(nullptr, SIM_ERR_ARG, "m must be >= 1");
+  if (n_replicas < 1) return fail(nullptr, SIM_ERR_ARG, "n_replicas must be >= 1");
+  if (replica_base < 0 || replica_base + (int64_t)n_replicas > (int64_t)1 << 32)
+    return fail(nullptr, SIM_ERR_ARG, "global replica ids must fit in 32 bits");
+  sim_status st = check_delay(nullptr, delay);
+  if (st != SIM_OK) return st;
+  if (!(eta == eta) || std::isinf(eta)) return fail(nullptr, SIM_ERR_ARG, "eta must be finite");
+
+  sim_problem prob{};
+  prob.model = SIM_NONE;
+  if (problem) prob = *problem;
+  if (prob.model != SIM_NONE) {
+    if ((int)prob.model < 0 || (int)prob.model > (int)SIM_MLP2) return fail(nullptr, SIM_ERR_ARG, "unknown model");
+    if (prob.n < 1 || prob.n > (int64_t)1 << 32) return fail(nullptr, SIM_ERR_ARG, "n must be in [1, 2^32]");
+    if (prob.d < 4 || prob.d % 4 != 0) return fail(nullptr, SIM_ERR_ARG, "d must be a positive multiple of 4");
+    if (!prob.X || (reinterpret_cast<uintptr_t>(prob.X) & 15u)) return fail(nullptr, SIM_ERR_ARG, "X must be a 16-byte aligned device pointer");
+    if (prob.model == SIM_LSQ && !prob.y) return fail(nullptr, SIM_ERR_ARG, "least squares needs y");
+    if (prob.model != SIM_LSQ && !prob.label) return fail(nullptr, SIM_ERR_ARG, "classification models need label");
+    if (prob.w_ref && (reinterpret_cast<uintptr_t>(prob.w_ref) & 15u)) return fail(nullptr, SIM_ERR_ARG, "w_ref must be 16-byte aligned");
+    if (prob.model == SIM_SOFTMAX || prob.model == SIM_MLP2) {
+      if (prob.n_classes < 2 || prob.n_classes > SIM_MAX_CLASSES) return fail(nullptr, SIM_ERR_ARG, "n_classes must be in [2, SIM_MAX_CLASSES]");
+    }
+    if (prob.model == SIM_SOFTMAX) {
+      const char* why = softmax_shape_unsupported(prob.d, prob.n_classes);
+      if (why) return fail(nullptr, SIM_ERR_ARG, why);
+    }
+    if (prob.model == SIM_MLP2) {
+      const char* why = mlp_shape_unsupported(prob.d, prob.hidden, prob.n_classes, m);
+      if (why) return fail(nullptr, SIM_ERR_ARG, why);
+    }
+    if ((prob.model == SIM_LSQ || prob.model == SIM_LOGISTIC) && prob.d > 8192)
+      return fail(nullptr, SIM_ERR_ARG, "d > 8192 is not supported by the linear-model kernel");
+  }
+
+  sim_handle* h = new (std::nothrow) sim_handle();
+  if (!h) return fail(nullptr, SIM_ERR_ALLOC, "host allocation failed");
+  h->prob = prob; h->P = P; h->K = K; h->variant = (int)variant; h->delay = delay; h->eta = eta;
+  h->m = m; h->seed = seed; h->R = n_replicas; h->replica_base = (uint32_t)replica_base;
+  h->stream = static_cast<cudaStream_t>(cuda_stream);
+  h->K_stride = K;
+  h->is_async = variant == SIM_KASYNC || variant == SIM_KBATCHASYNC;
+  h->n_slots = h->is_async ? P + 2 : 0;
+  h->n_params = model_params(prob);
+
+  cudaError_t e = cudaGetDevice(&h->device);
+  const size_t RP = (size_t)h->R * P;
+  if (e == cudaSuccess) e = dev_alloc(&h->s, RP, h->stream);
+  if (e == cudaSuccess) e = dev_alloc(&h->tau, RP, h->stream);
+  if (e == cudaSuccess) e = dev_alloc(&h->f, RP, h->stream);
+  if (e == cudaSuccess) e = dev_alloc(&h->wslot, RP, h->stream);
+  if (e == cudaSuccess) e = dev_alloc(&h->cur_slot, (size_t)h->R, h->stream);
+  if (e == cudaSuccess) e = dev_alloc(&h->begin_slot, (size_t)h->R, h->stream);
+  if (e == cudaSuccess) e = dev_alloc(&h->clock, (size_t)h->R, h->stream);
+  if (e == cudaSuccess) e = dev_alloc(&h->err, 1, h->stream);
+  if (e == cudaSuccess && h->n_params > 0) {
+    if (h->is_async) e = dev_alloc(&h->pool, (size_t)h->R * h->n_slots * h->n_params, h->stream);
+    else e = dev_alloc(&h->w_state, (size_t)h->R * h->n_params, h->stream);
+  }
+  if (e == cudaSuccess && prob.model == SIM_MLP2) e = mlp_scratch_alloc(h->mlp, prob.d, prob.hidden, prob.n_classes, m, P, h->R, h->n_slots, h->is_async, h->stream);
+  if (e != cudaSuccess) {
+    const sim_status code = e == cudaErrorMemoryAllocation ? SIM_ERR_ALLOC : SIM_ERR_CUDA;
+    std::string msg = std::string("sim_create: ") + cudaGetErrorString(e);
+    free_all(h);
+    delete h;
+    cudaGetLastError();
+    return fail(nullptr, code, msg);
+  }
+  *out = h;
+  return SIM_OK;
+}
+
+sim_status sim_set_params(sim_handle* h, const float* w0) {
+  if (!h) return fail(nullptr, SIM_ERR_ARG, "handle is NULL");
+  if (!w0) return fail(h, SIM_ERR_ARG, "w0 is NULL");
+  if (h->n_updates > 0) return fail(h, SIM_ERR_STATE, "sim_set_params is only allowed before the first sim_run");
+  if (h->n_params == 0) return SIM_OK;
+  float* dst = h->is_async ? h->pool : h->w_state;
+  const long long stride = h->is_async ? (long long)h->n_slots * h->n_params : h->n_params;
+  broadcast_params_kernel<<<1184, 256, 0, h->stream>>>(w0, dst, h->n_params, stride, h->R);
+  CUDA_TRY(h, cudaGetLastError());
+  if (h->prob.model == SIM_MLP2) {
+    sim_status st = mlp_after_set_params(h->mlp, dst, stride, h->R, h->stream) == cudaSuccess ? SIM_OK : SIM_ERR_CUDA;
+    if (st != SIM_OK) return fail(h, st, "mlp parameter preparation failed");
+  }
+  // the caller's buffer is read by enqueued work: finish it before returning
+  CUDA_TRY(h, cudaStreamSynchronize(h->stream));
+  return SIM_OK;
+}
+
+sim_status sim_set_adasync(sim_handle* h, int32_t K0, double t_interval) {
+  if (!h) return fail(nullptr, SIM_ERR_ARG, "handle is NULL");
+  if (h->n_updates > 0 || h->cap > 0) return fail(h, SIM_ERR_STATE, "sim_set_adasync is only allowed before sim_reserve / sim_run");
+  if (t_interval > 0.0) {
+    if (K0 < 1 || K0 > h->P) return fail(h, SIM_ERR_ARG, "K0 must be in [1, P]");
+    h->K0 = K0; h->t_interval = t_interval; h->K_stride = h->P;
+  } else {
+    h->K0 = 0; h->t_interval = 0.0; h->K_stride = h->K;
+  }
+  return SIM_OK;
+}
+
+sim_status sim_set_tuning(sim_handle* h, int32_t stages) {
+  if (!h) return fail(nullptr, SIM_ERR_ARG, "handle is NULL");
+  if (stages < 0 || stages == 1 || stages > 8) return fail(h, SIM_ERR_ARG, "stages must be 0 (automatic) or in [2, 8]");
+  h->tune_stages = stages;
+  return SIM_OK;
+}
+
+sim_status sim_reserve(sim_handle* h, int64_t total_updates) {
+  if (!h) return fail(nullptr, SIM_ERR_ARG, "handle is NULL");
+  if (total_updates < 0) return fail(h, SIM_ERR_ARG, "total_updates must be >= 0");
+  return ensure_capacity(h, total_updates);
+}
+
+sim_status sim_run(sim_handle* h, int64_t iters) {
+  if (!h) return fail(nullptr, SIM_ERR_ARG, "handle is NULL");
+  if (iters < 0) return fail(h, SIM_ERR_ARG, "iters must be >= 0");
+  if (h->poisoned) return fail(h, SIM_ERR_STATE, "the handle failed earlier and cannot run");
+  if (iters == 0) return SIM_OK;
+  if (h->n_updates + iters > (1ll << 31)) return fail(h, SIM_ERR_ARG, "more than 2^31 updates");
+  sim_status st = ensure_capacity(h, h->n_updates + iters);
+  if (st != SIM_OK) return st;
+
+  ScheduleArgs sa{};
+  sa.variant = h->variant; sa.P = h->P; sa.K_fixed = h->K; sa.K0 = h->K0; sa.t_interval = h->t_interval;
+  sa.law.shifted = h->delay.kind == SIM_DELAY_SHIFTED_EXP; sa.law.mu = h->delay.mu; sa.law.shift = h->delay.shift;
+  sa.seed = h->seed; sa.R = h->R; sa.replica_base = h->replica_base;
+  sa.j0 = h->n_updates; sa.iters = iters; sa.cap = h->cap; sa.K_stride = h->K_stride; sa.n_slots = h->n_slots;
+  sa.s = h->s; sa.tau = h->tau; sa.f = h->f; sa.wslot = h->wslot; sa.cur_slot = h->cur_slot;
+  sa.begin_slot = h->begin_slot; sa.clock = h->clock;
+  sa.t = h->tr.t; sa.K_used = h->tr.K_used; sa.worker = h->tr.worker; sa.stale = h->tr.stale; sa.seq = h->tr.seq;
+  sa.snap_slot = h->tr.snap_slot; sa.new_slot = h->tr.new_slot; sa.err = h->err;
+  schedule_kernel<<<(h->R + 3) / 4, 128, 0, h->stream>>>(sa);
+  CUDA_TRY(h, cudaGetLastError());
+
+  if (h->prob.model != SIM_NONE) {
+    NumericArgs a{};
+    a.X = h->prob.X;
+    a.y = h->prob.model == SIM_LSQ ? static_cast<const void*>(h->prob.y) : static_cast<const void*>(h->prob.label);
+    a.w_ref = h->prob.w_ref; a.n = (uint64_t)h->prob.n; a.d = h->prob.d; a.m = h->m; a.model = (int)h->prob.model;
+    a.n_classes = h->prob.n_classes; a.eta = h->eta; a.seed = h->seed; a.replica_base = h->replica_base; a.R = h->R;
+    a.j0 = h->n_updates; a.iters = iters; a.cap = h->cap; a.K_stride = h->K_stride; a.is_async = h->is_async ? 1 : 0;
+    a.n_slots = h->n_slots; a.n_params = h->n_params;
+    a.K_used = h->tr.K_used; a.worker = h->tr.worker; a.seq = h->tr.seq; a.snap_slot = h->tr.snap_slot;
+    a.new_slot = h->tr.new_slot; a.begin_slot = h->begin_slot; a.loss = h->tr.loss; a.dist2 = h->tr.dist2;
+    a.w_state = h->w_state; a.pool = h->pool; a.err = h->err;
+    const char* why = nullptr;
+    cudaError_t ce = cudaSuccess;
+    switch (h->prob.model) {
+      case SIM_LSQ: case SIM_LOGISTIC: st = run_linear1(h, a); break;
+      case SIM_SOFTMAX:
+        ce = run_softmax(a, h->tune_stages, h->stream, &why);
+        st = why ? fail(h, SIM_ERR_ARG, why) : SIM_OK;
+        break;
+      case SIM_MLP2:
+        ce = run_mlp(a, h->mlp, h->prob.hidden, h->P, h->stream, &why);
+        st = why ? fail(h, SIM_ERR_ARG, why) : SIM_OK;
+        break;
+      default: st = fail(h, SIM_ERR_ARG, "unknown model");
+    }
+    if (ce != cudaSuccess) st = fail(h, SIM_ERR_CUDA, std::string("numeric kernel launch: ") + cudaGetErrorString(ce));
+    if (st != SIM_OK) { h->poisoned = true; return st; }
+  }
+  h->n_updates += iters;
+  return SIM_OK;
+}
+
+sim_status sim_trace_size(const sim_handle* h, int64_t* n_updates, int32_t* K_max) {
+  if (!h) return fail(nullptr, SIM_ERR_ARG, "handle is NULL");
+  sim_status st = device_error(h);
+  if (st != SIM_OK) return st;
+  if (n_updates) *n_updates = h->n_updates;
+  if (K_max) *K_max = h->K_stride;
+  return SIM_OK;
+}
+
+sim_status sim_get_trace(const sim_handle* h, double* t, float* loss, float* dist2, uint16_t* K_used,
+                         uint16_t* worker, uint32_t* stale, uint32_t* seq) {
+  if (!h) return fail(nullptr, SIM_ERR_ARG, "handle is NULL");
+  sim_status st = device_error(h);
+  if (st != SIM_OK) return st;
+  const long long J = h->n_updates;
+  if (J == 0) return SIM_OK;
+  const size_t Ks = (size_t)h->K_stride;
+  auto copy = [&](void* dst, const void* src, size_t elem) -> cudaError_t {
+    if (!dst) return cudaSuccess;
+    return cudaMemcpy2DAsync(dst, (size_t)J * elem, src, (size_t)h->cap * elem, (size_t)J * elem, h->R,
+                             cudaMemcpyDeviceToDevice, h->stream);
+  };
+  CUDA_TRY(h, copy(t, h->tr.t, 8));
+  CUDA_TRY(h, copy(loss, h->tr.loss, 4));
+  CUDA_TRY(h, copy(dist2, h->tr.dist2, 4));
+  CUDA_TRY(h, copy(K_used, h->tr.K_used, 2));
+  CUDA_TRY(h, copy(worker, h->tr.worker, 2 * Ks));
+  CUDA_TRY(h, copy(stale, h->tr.stale, 4 * Ks));
+  CUDA_TRY(h, copy(seq, h->tr.seq, 4 * Ks));
+  CUDA_TRY(h, cudaStreamSynchronize(h->stream));
+  return SIM_OK;
+}
+
+sim_status sim_get_params(const sim_handle* h, float* w) {
+  if (!h) return fail(nullptr, SIM_ERR_ARG, "handle is NULL");
+  if (!w) return fail(h, SIM_ERR_ARG, "w is NULL");
+  sim_status st = device_error(h);
+  if (st != SIM_OK) return st;
+  if (h->n_params == 0) return SIM_OK;
+  if (h->is_async) {
+    gather_params_kernel<<<1184, 256, 0, h->stream>>>(h->pool, h->cur_slot, w, h->n_params, h->n_slots, h->R);
+    CUDA_TRY(h, cudaGetLastError());
+  } else {
+    CUDA_TRY(h, cudaMemcpyAsync(w, h->w_state, (size_t)h->R * h->n_params * sizeof(float), cudaMemcpyDeviceToDevice, h->stream));
+  }
+  CUDA_TRY(h, cudaStreamSynchronize(h->stream));
+  return SIM_OK;
+}
+
+int64_t sim_n_params(const sim_handle* h) { return h ? h->n_params : 0; }
+
+const char* sim_last_error(const sim_handle* h) { return h ? h->last_error.c_str() : g_last_error.c_str(); }
+
+void sim_destroy(sim_handle* h) {
+  if (!h) return;
+  cudaStreamSynchronize(h->stream);
+  free_all(h);
+  delete h;
+}
+
+sim_status sim_draw_delays(sim_delay delay, uint64_t seed, int64_t replica_base, int32_t n_replicas,
+                           int32_t P, int32_t n_seq, double* out, void* cuda_stream) {
+  sim_status st = check_delay(nullptr, delay);
+  if (st != SIM_OK) return st;
+  if (!out || n_replicas < 1 || P < 1 || n_seq < 1 || replica_base < 0 || replica_base + (int64_t)n_replicas > (int64_t)1 << 32)
+    return fail(nullptr, SIM_ERR_ARG, "sim_draw_delays: bad argument");
+  DelayLaw law{delay.kind == SIM_DELAY_SHIFTED_EXP, delay.mu, delay.shift};
+  draw_delays_kernel<<<592, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(law, seed, (uint32_t)replica_base, n_replicas, P, n_seq, out);
+  CUDA_TRY(nullptr, cudaGetLastError());
+  return SIM_OK;
+}
+
+sim_status sim_draw_indices(uint64_t seed, int64_t replica_base, int32_t n_replicas, int32_t P,
+                            int32_t n_seq, int64_t n, int32_t m, uint32_t* out, void* cuda_stream) {
+  if (!out || n_replicas < 1 || P < 1 || n_seq < 1 || m < 1 || n < 1 || n > (int64_t)1 << 32 || replica_base < 0 ||
+      replica_base + (int64_t)n_replicas > (int64_t)1 << 32)
+    return fail(nullptr, SIM_ERR_ARG, "sim_draw_indices: bad argument");
+  draw_indices_kernel<<<592, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(seed, (uint32_t)replica_base, n_replicas, P, n_seq, (uint64_t)n, m, out);
+  CUDA_TRY(nullptr, cudaGetLastError());
+  return SIM_OK;
+}
+
+sim_status sim_simulate_host(const sim_problem* problem, int32_t P, int32_t K, sim_variant variant,
+                             sim_delay delay, float eta, int32_t m, uint64_t seed, int32_t n_replicas,
+                             int64_t replica_base, const float* w0, int32_t K0, double t_interval,
+                             int64_t iters, double* t, float* loss, float* dist2, uint16_t* K_used,
+                             uint16_t* worker, uint32_t* stale, uint32_t* seq, float* w_final) {
+  if (iters < 0) return fail(nullptr, SIM_ERR_ARG, "iters must be >= 0");
+  sim_problem dp{};
+  dp.model = SIM_NONE;
+  std::vector<void*> owned;
+  sim_handle* h = nullptr;
+  sim_status st = SIM_OK;
+  std::string msg;
+  auto up = [&](const void* src, size_t bytes, void** dst) -> bool {
+    *dst = nullptr;
+    if (!src || bytes == 0) return true;
+    cudaError_t e = cudaMalloc(dst, bytes);
+    if (e == cudaSuccess) { owned.push_back(*dst); e = cudaMemcpyAsync(*dst, src, bytes, cudaMemcpyHostToDevice, nullptr); }
+    if (e != cudaSuccess) { st = e == cudaErrorMemoryAllocation ? SIM_ERR_ALLOC : SIM_ERR_CUDA; msg = cudaGetErrorString(e); return false; }
+    return true;
+  };
+  auto down = [&](void* host, size_t bytes, auto getter) -> bool {
+    if (!host || bytes == 0) return true;
+    void* dev = nullptr;
+    cudaError_t e = cudaMalloc(&dev, bytes);
+    if (e != cudaSuccess) { st = SIM_ERR_ALLOC; msg = cudaGetErrorString(e); return false; }
+    owned.push_back(dev);
+    st = getter(dev);
+    if (st != SIM_OK) { msg = sim_last_error(h); return false; }
+    e = cudaMemcpy(host, dev, bytes, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) { st = SIM_ERR_CUDA; msg = cudaGetErrorString(e); return false; }
+    return true;
+  };
+  do {
+    void* dw0 = nullptr;
+    long long np = 0;
+    if (problem && problem->model != SIM_NONE) {
+      dp = *problem;
+      if (dp.n < 1 || dp.d < 1 || !dp.X) { st = SIM_ERR_ARG; msg = "bad problem"; break; }
+      np = model_params(dp);
+      void *X, *y, *lab, *wr;
+      if (!up(problem->X, (size_t)dp.n * dp.d * 4, &X)) break;
+      if (!up(problem->y, (size_t)dp.n * 4, &y)) break;
+      if (!up(problem->label, (size_t)dp.n * 4, &lab)) break;
+      if (!up(problem->w_ref, (size_t)np * 4, &wr)) break;
+      dp.X = (const float*)X; dp.y = (const float*)y; dp.label = (const int32_t*)lab; dp.w_ref = (const float*)wr;
+      if (!up(w0, (size_t)np * 4, &dw0)) break;
+    }
+    st = sim_create(&dp, P, K, variant, delay, eta, m, seed, n_replicas, replica_base, nullptr, &h);
+    if (st != SIM_OK) { msg = g_last_error; break; }
+    if (t_interval > 0.0 && (st = sim_set_adasync(h, K0, t_interval)) != SIM_OK) { msg = sim_last_error(h); break; }
+    if (dw0 && (st = sim_set_params(h, (const float*)dw0)) != SIM_OK) { msg = sim_last_error(h); break; }
+    if ((st = sim_run(h, iters)) != SIM_OK) { msg = sim_last_error(h); break; }
+    const size_t RJ = (size_t)n_replicas * iters, Ks = (size_t)h->K_stride;
+    if (!down(t, RJ * 8, [&](void* p) { return sim_get_trace(h, (double*)p, 0, 0, 0, 0, 0, 0); })) break;
+    if (!down(loss, RJ * 4, [&](void* p) { return sim_get_trace(h, 0, (float*)p, 0, 0, 0, 0, 0); })) break;
+    if (!down(dist2, RJ * 4, [&](void* p) { return sim_get_trace(h, 0, 0, (float*)p, 0, 0, 0, 0); })) break;
+    if (!down(K_used, RJ * 2, [&](void* p) { return sim_get_trace(h, 0, 0, 0, (uint16_t*)p, 0, 0, 0); })) break;
+    if (!down(worker, RJ * Ks * 2, [&](void* p) { return sim_get_trace(h, 0, 0, 0, 0, (uint16_t*)p, 0, 0); })) break;
+    if (!down(stale, RJ * Ks * 4, [&](void* p) { return sim_get_trace(h, 0, 0, 0, 0, 0, (uint32_t*)p, 0); })) break;
+    if (!down(seq, RJ * Ks * 4, [&](void* p) { return sim_get_trace(h, 0, 0, 0, 0, 0, 0, (uint32_t*)p); })) break;
+    if (np > 0 && !down(w_final, (size_t)n_replicas * np * 4, [&](void* p) { return sim_get_params(h, (float*)p); })) break;
+    if (st == SIM_OK) st = device_error(h);
+    if (st != SIM_OK) msg = sim_last_error(h);
+  } while (0);
+  if (h) sim_destroy(h); else cudaDeviceSynchronize();
+  for (void* p : owned) cudaFree(p);
+  if (st != SIM_OK) return fail(nullptr, st, "sim_simulate_host: " + msg);
+  return SIM_OK;
+}
+
+}  // extern "C"

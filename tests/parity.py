@@ -1,0 +1,67 @@
+"""Helpers shared by the GPU parity tests: run the library and the CPU oracle on the same seeded
+inputs and compare.  Integers and fp64 times must be bit-identical; fp32 parameters must agree
+to 1e-5 in relative 2-norm at every compared step and per-update losses to 1e-5 relative."""
+import numpy as np
+import torch
+
+from oracle import core
+from oracle.sim import OracleReplica
+
+PARAM_RTOL = 1e-5
+LOSS_RTOL = 1e-5
+
+
+def to_device(data):
+    out = {"model": data["model"], "n_classes": data.get("n_classes", 1), "hidden": data.get("hidden", 0)}
+    out["X"] = torch.from_numpy(data["X"]).cuda()
+    out["y"] = torch.from_numpy(data["y"]).cuda()
+    return out
+
+
+def assert_schedule_equal(gpu, ora, rows=None):
+    """gpu: trace dict from the library; ora: dict from oracle BulkSchedule.run (same shapes)."""
+    for k in ("t", "K", "worker", "stale", "seq"):
+        a, b = gpu[k], ora[k]
+        if rows is not None:
+            a = a[rows]
+        if k == "t":
+            a, b = a.view(np.int64), b.view(np.int64)     # bit-exact fp64
+        assert a.shape == b.shape, (k, a.shape, b.shape)
+        if not np.array_equal(a, b):
+            bad = np.argwhere(a != b)[0]
+            raise AssertionError("schedule mismatch in %s at %s: gpu %s oracle %s" % (k, bad, a[tuple(bad)], b[tuple(bad)]))
+
+
+def oracle_schedule(wl_kw, variant, K, R, J, replica_base=0, K0=0, t_interval=0.0, chunks=None):
+    b = core.BulkSchedule(variant, wl_kw["P"], K, wl_kw["delay_kind"], wl_kw["mu"], wl_kw["shift"], wl_kw["seed"], R,
+                          replica_base=replica_base, K0=K0, t_interval=t_interval)
+    return b.run(J)
+
+
+def oracle_replica(data, w0, r, *, P, K, variant, delay_kind, mu, shift, eta, m, seed, w_ref=None, K0=0, t_interval=0.0):
+    return OracleReplica(model=data["model"], X=data["X"], y=data["y"], w0=w0, P=P, K=K, variant=variant,
+                         delay_kind=delay_kind, mu=mu, shift=shift, eta=eta, m=m, seed=seed, replica=r,
+                         n_classes=data.get("n_classes", 1), hidden=data.get("hidden", 0), w_ref=w_ref,
+                         K0=K0, t_interval=t_interval)
+
+
+def rel_norm(a, b):
+    a, b = np.asarray(a, np.float64), np.asarray(b, np.float64)
+    nb = np.linalg.norm(b)
+    return np.linalg.norm(a - b) / (nb if nb > 0 else 1.0)
+
+
+def assert_params_close(w_gpu, w_ora, what="", rtol=PARAM_RTOL):
+    e = rel_norm(w_gpu, w_ora)
+    assert e <= rtol, "%s: |w_gpu - w_oracle| / |w_oracle| = %.3g > %.1g" % (what, e, rtol)
+    return e
+
+
+def assert_loss_close(l_gpu, l_ora, what="", rtol=LOSS_RTOL):
+    """Per update: |dL| <= rtol * max(|L_oracle|, 1e-6 * L_0), L_0 the first update's loss."""
+    l_gpu, l_ora = np.asarray(l_gpu, np.float64), np.asarray(l_ora, np.float64)
+    floor = 1e-6 * abs(l_ora.flat[0])
+    err = np.abs(l_gpu - l_ora) / np.maximum(np.abs(l_ora), floor)
+    assert err.max() <= rtol, "%s: loss relative error %.3g at update %d (gpu %.9g oracle %.9g)" % (
+        what, err.max(), int(err.argmax()), l_gpu.flat[err.argmax()], l_ora.flat[err.argmax()])
+    return err.max()
