@@ -168,6 +168,40 @@ sim_status sim_simulate_host(const sim_problem* problem, int32_t P, int32_t K, s
                              int64_t iters, double* t, float* loss, float* dist2, uint16_t* K_used,
                              uint16_t* worker, uint32_t* stale, uint32_t* seq, float* w_final);
 
+/*
+ * Clock-only simulation for callers that cannot allocate device memory.  (The paper has no
+ * counterpart for this entry point: it exists for the sake of the library's users, not of the
+ * method.)
+ *
+ * Who needs it: code that must not call cudaMalloc while it runs - a service loop in which an
+ * allocation would stall every stream of the device, a process whose device memory is owned by a
+ * pool that forbids side allocations, a thread sharing the GPU with a job that has already taken
+ * the memory it may use.  sim_create / sim_run allocate worker state and a trace; this call
+ * allocates nothing, neither directly nor through any library.  It runs the arrival process of
+ * Section 2.2 (same variants, delays, growing-K rule and random streams as a SIM_NONE handle,
+ * bit for bit) for `iters` updates from update 0 and writes the schedule straight into the
+ * caller's DEVICE buffers, all five required:
+ *   t [R][iters], K_used [R][iters], worker / stale / seq [R][iters][K_max],
+ *   K_max = K, or P when t_interval > 0 (then K0 is the first K and K is ignored).
+ * The per-replica worker state lives in one fixed array inside the library image
+ * (SIM_NOALLOC_SCRATCH_BYTES of device memory on every GPU that loads the library, held until the
+ * process exits), which bounds the problem: n_replicas <= SIM_NOALLOC_MAX_REPLICAS and
+ * n_replicas * P <= SIM_NOALLOC_MAX_REPLICA_WORKERS; larger requests return SIM_ERR_ARG and launch
+ * nothing.  The first call on each device looks up the array's device address; make that first
+ * call outside any stream capture.  All calls on a device share the array and each call clears
+ * the part it uses before it starts, so two calls whose GPU work overlaps (different streams or
+ * threads) race: serialise them.  Work is enqueued on `cuda_stream`; the call does not wait for
+ * it.  On failure sim_noalloc_last_error() describes the cause (per host thread).
+ */
+#define SIM_NOALLOC_MAX_REPLICAS 4096
+#define SIM_NOALLOC_MAX_REPLICA_WORKERS 65536
+#define SIM_NOALLOC_SCRATCH_BYTES (1088 * 1024)
+sim_status sim_schedule_noalloc(int32_t P, int32_t K, sim_variant variant, sim_delay delay, uint64_t seed,
+                                int64_t replica_base, int32_t n_replicas, int32_t K0, double t_interval,
+                                int64_t iters, double* t, uint16_t* K_used, uint16_t* worker,
+                                uint32_t* stale, uint32_t* seq, void* cuda_stream);
+const char* sim_noalloc_last_error(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -21,7 +21,8 @@ STATUS = {0: "SIM_OK", 1: "SIM_ERR_ARG", 2: "SIM_ERR_ALLOC", 3: "SIM_ERR_CUDA", 
 
 EXPORTS = ["sim_create", "sim_set_params", "sim_set_adasync", "sim_set_tuning", "sim_reserve", "sim_run",
            "sim_trace_size", "sim_get_trace", "sim_get_params", "sim_n_params", "sim_last_error",
-           "sim_destroy", "sim_draw_delays", "sim_draw_indices", "sim_simulate_host"]
+           "sim_destroy", "sim_draw_delays", "sim_draw_indices", "sim_simulate_host", "sim_schedule_noalloc",
+           "sim_noalloc_last_error"]
 
 
 class SimProblem(C.Structure):
@@ -66,8 +67,11 @@ def _load():
     L.sim_draw_indices.argtypes = [u64, i64, i32, i32, i32, i64, i32, vp, vp]
     L.sim_simulate_host.argtypes = [C.POINTER(SimProblem), i32, i32, C.c_int, SimDelay, C.c_float, i32, u64,
                                     i32, i64, vp, i32, dbl, i64] + [vp] * 8
+    L.sim_schedule_noalloc.argtypes = [i32, i32, C.c_int, SimDelay, u64, i64, i32, i32, dbl, i64] + [vp] * 6
+    L.sim_noalloc_last_error.argtypes = []
+    L.sim_noalloc_last_error.restype = C.c_char_p
     for name in EXPORTS:
-        if name not in ("sim_n_params", "sim_last_error", "sim_destroy"):
+        if name not in ("sim_n_params", "sim_last_error", "sim_destroy", "sim_noalloc_last_error"):
             getattr(L, name).restype = C.c_int
     return L
 
@@ -195,6 +199,21 @@ def draw_indices(seed, replica_base, n_replicas, P, n_seq, n, m):
     _check(lib.sim_draw_indices(seed, replica_base, n_replicas, P, n_seq, n, m, _ptr(out),
                                 _stream_ptr(torch.cuda.current_stream())))
     return out.cpu().numpy()
+
+
+def schedule_noalloc(out, *, P, K, variant, delay_kind, mu, shift=0.0, seed, n_replicas, iters, replica_base=0,
+                     K0=0, t_interval=0.0, stream=None):
+    """Clock-only simulation through the entry point that allocates nothing: the caller brings
+    the five output tensors (`out`: t, K, worker, stale, seq on the device, shaped as in
+    Simulation.trace) because the library may not create them.  For callers that cannot call
+    cudaMalloc; the worker state sits in a fixed array inside the library, so sizes are capped and
+    calls on one device must not overlap."""
+    st = lib.sim_schedule_noalloc(P, K, VARIANTS[variant], SimDelay(DELAYS[delay_kind], mu, shift), seed,
+                                  replica_base, n_replicas, K0, t_interval, iters,
+                                  *[_ptr(out[k]) for k in ("t", "K", "worker", "stale", "seq")],
+                                  _stream_ptr(stream))
+    if st != 0:
+        raise SimError(st, lib.sim_noalloc_last_error().decode())
 
 
 def simulate_host(data, *, P, K, variant, delay_kind, mu, shift=0.0, eta, m, seed, n_replicas, iters,
