@@ -46,6 +46,7 @@ struct sim_handle {
   double t_interval = 0.0;
   int K_stride = 0;
   bool is_async = false;
+  bool uses_pool = false;     // parameters live in a version pool (asynchronous variants, and the MLP always)
   int n_slots = 0;
   long long n_params = 0;
   long long n_updates = 0, cap = 0;
@@ -267,7 +268,8 @@ sim_status sim_create(const sim_problem* problem, int32_t P, int32_t K, sim_vari
   h->stream = static_cast<cudaStream_t>(cuda_stream);
   h->K_stride = K;
   h->is_async = variant == SIM_KASYNC || variant == SIM_KBATCHASYNC;
-  h->n_slots = h->is_async ? P + 2 : 0;
+  h->uses_pool = h->is_async || prob.model == SIM_MLP2;
+  h->n_slots = h->is_async ? P + 2 : (prob.model == SIM_MLP2 ? 2 : 0);
   h->n_params = model_params(prob);
 
   cudaError_t e = cudaGetDevice(&h->device);
@@ -281,10 +283,9 @@ sim_status sim_create(const sim_problem* problem, int32_t P, int32_t K, sim_vari
   if (e == cudaSuccess) e = dev_alloc(&h->clock, (size_t)h->R, h->stream);
   if (e == cudaSuccess) e = dev_alloc(&h->err, 1, h->stream);
   if (e == cudaSuccess && h->n_params > 0) {
-    if (h->is_async) e = dev_alloc(&h->pool, (size_t)h->R * h->n_slots * h->n_params, h->stream);
+    if (h->uses_pool) e = dev_alloc(&h->pool, (size_t)h->R * h->n_slots * h->n_params, h->stream);
     else e = dev_alloc(&h->w_state, (size_t)h->R * h->n_params, h->stream);
   }
-  if (e == cudaSuccess && prob.model == SIM_MLP2) e = mlp_scratch_alloc(h->mlp, prob.d, prob.hidden, prob.n_classes, m, P, h->R, h->n_slots, h->is_async, h->stream);
   if (e != cudaSuccess) {
     const sim_status code = e == cudaErrorMemoryAllocation ? SIM_ERR_ALLOC : SIM_ERR_CUDA;
     std::string msg = std::string("sim_create: ") + cudaGetErrorString(e);
@@ -302,14 +303,10 @@ sim_status sim_set_params(sim_handle* h, const float* w0) {
   if (!w0) return fail(h, SIM_ERR_ARG, "w0 is NULL");
   if (h->n_updates > 0) return fail(h, SIM_ERR_STATE, "sim_set_params is only allowed before the first sim_run");
   if (h->n_params == 0) return SIM_OK;
-  float* dst = h->is_async ? h->pool : h->w_state;
-  const long long stride = h->is_async ? (long long)h->n_slots * h->n_params : h->n_params;
+  float* dst = h->uses_pool ? h->pool : h->w_state;
+  const long long stride = h->uses_pool ? (long long)h->n_slots * h->n_params : h->n_params;
   broadcast_params_kernel<<<1184, 256, 0, h->stream>>>(w0, dst, h->n_params, stride, h->R);
   CUDA_TRY(h, cudaGetLastError());
-  if (h->prob.model == SIM_MLP2) {
-    sim_status st = mlp_after_set_params(h->mlp, dst, stride, h->R, h->stream) == cudaSuccess ? SIM_OK : SIM_ERR_CUDA;
-    if (st != SIM_OK) return fail(h, st, "mlp parameter preparation failed");
-  }
   // the caller's buffer is read by enqueued work: finish it before returning
   CUDA_TRY(h, cudaStreamSynchronize(h->stream));
   return SIM_OK;
@@ -381,7 +378,14 @@ sim_status sim_run(sim_handle* h, int64_t iters) {
         st = why ? fail(h, SIM_ERR_ARG, why) : SIM_OK;
         break;
       case SIM_MLP2:
-        ce = run_mlp(a, h->mlp, h->prob.hidden, h->P, h->stream, &why);
+        if (!h->mlp.Xq) {   // first run: bf16 copy of the data, per-update scratch, bf16 shadow of the initial W1
+          ce = mlp_scratch_alloc(h->mlp, h->prob.X, h->prob.n, h->prob.d, h->prob.hidden, h->prob.n_classes, h->m,
+                                 h->K_stride, h->R, h->n_slots, h->stream);
+          if (ce == cudaSuccess) ce = mlp_after_set_params(h->mlp, h->pool, h->n_params, h->stream);
+        }
+        if (ce == cudaSuccess) ce = run_mlp(a, h->mlp, h->P, h->stream, &why);
+        if (ce == cudaSuccess && !h->is_async)   // synchronous variants ping-pong between two slots
+          ce = cudaMemsetAsync(h->cur_slot, (int)((h->n_updates + iters) & 1), (size_t)h->R, h->stream);
         st = why ? fail(h, SIM_ERR_ARG, why) : SIM_OK;
         break;
       default: st = fail(h, SIM_ERR_ARG, "unknown model");
@@ -432,7 +436,7 @@ sim_status sim_get_params(const sim_handle* h, float* w) {
   sim_status st = device_error(h);
   if (st != SIM_OK) return st;
   if (h->n_params == 0) return SIM_OK;
-  if (h->is_async) {
+  if (h->uses_pool) {
     gather_params_kernel<<<1184, 256, 0, h->stream>>>(h->pool, h->cur_slot, w, h->n_params, h->n_slots, h->R);
     CUDA_TRY(h, cudaGetLastError());
   } else {
