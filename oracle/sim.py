@@ -52,7 +52,7 @@ class OracleReplica:
         self.snap = [self.w] * P         # the parameters worker i last fetched
         self.f = [0.0] * P               # absolute end time of worker i's running task
         self.started = False
-        self.trace = {k: [] for k in ("t", "K", "worker", "stale", "seq", "loss", "dist2")}
+        self.trace = {k: [] for k in ("t", "K", "worker", "stale", "seq", "loss", "dist2", "gnorm")}
 
     # -- random quantities ----------------------------------------------------------------
     def _delay(self, i):
@@ -93,6 +93,7 @@ class OracleReplica:
                 loss += f_sum
             self.w = (self.w.astype(np.float64) - (self.eta / K) * total).astype(np.float32)
             tr["loss"].append(np.float32(loss / (K * self.m)))
+            tr["gnorm"].append(float(np.linalg.norm(total)) / K)     # |averaged gradient| of this update
             if self.w_ref is not None:
                 dv = self.w.astype(np.float64) - self.w_ref
                 tr["dist2"].append(np.float32(dv @ dv))
@@ -172,7 +173,8 @@ class OracleReplica:
                "worker": np.full((J, Ks), 0xFFFF, np.uint16),
                "stale": np.full((J, Ks), 0xFFFFFFFF, np.uint32),
                "seq": np.full((J, Ks), 0xFFFFFFFF, np.uint32),
-               "loss": np.array(tr["loss"], np.float32), "dist2": np.array(tr["dist2"], np.float32)}
+               "loss": np.array(tr["loss"], np.float32), "dist2": np.array(tr["dist2"], np.float32),
+               "gnorm": np.array(tr["gnorm"], np.float64)}
         for j in range(J):
             k = tr["K"][j]
             out["worker"][j, :k] = tr["worker"][j]

@@ -302,8 +302,11 @@ __global__ void __launch_bounds__(NT) linear1_kernel(NumericArgs a) {
         } else {  // logistic, label b in {0,1}: f = softplus(z) - b z, df/dz = sigmoid(z) - b
           const float b = (float)(int)yraw;
           const float ez = expf(-fabsf(z));
-          const float sig = z >= 0.f ? 1.f / (1.f + ez) : ez / (1.f + ez);
-          aq[q] = sig - b;
+          // sigmoid(z) - b without cancellation: sigma - 1 is formed directly for b = 1
+          const float inv = 1.f / (1.f + ez);
+          const float sig = z >= 0.f ? inv : ez * inv;
+          const float sig_m1 = z >= 0.f ? -ez * inv : -inv;
+          aq[q] = b != 0.f ? sig_m1 : sig;
           loss_acc += fmaxf(z, 0.f) + log1pf(ez) - b * z;
         }
       }

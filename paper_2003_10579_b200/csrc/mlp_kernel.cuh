@@ -305,19 +305,29 @@ __global__ void __launch_bounds__(256, 1) mlp_forward_kernel(MlpArgs g) {
       z[c] = c < C ? s + b2[c] : -INFINITY;
       zmax = fmaxf(zmax, z[c]);
     }
-    float ssum = 0.f, zlab = 0.f;
+    // exponentials without the maximal class (its term is exactly 1): log(1 + s) and
+    // p_max - 1 = -s / (1 + s) stay accurate for samples classified with a wide margin
+    int cmax = 0;
 #pragma unroll
-    for (int c = 0; c < 16; ++c) { z[c] = c < C ? expf(z[c] - zmax) : 0.f; ssum += z[c]; }
+    for (int c = 15; c >= 0; --c) if (c < C && z[c] == zmax) cmax = c;
+    float zl = 0.f;
+#pragma unroll
+    for (int c = 0; c < 16; ++c) if (c == lab) zl = z[c];
+    float sexcl = 0.f;
+#pragma unroll
+    for (int c = 0; c < 16; ++c) { z[c] = (c < C && c != cmax) ? expf(z[c] - zmax) : 0.f; sexcl += z[c]; }
+    const float ssum = 1.f + sexcl;
 #pragma unroll
     for (int c = 0; c < 16; ++c) {
-      const float p = z[c] / ssum;
-      const float dl = c < C ? p - (c == lab ? 1.f : 0.f) : 0.f;
+      float dl = 0.f;
+      if (c < C) {
+        if (c == cmax) dl = c == lab ? -sexcl / ssum : 1.f / ssum;
+        else dl = z[c] / ssum - (c == lab ? 1.f : 0.f);
+      }
       d2_s[row * 16 + c] = dl;
       sc.D2[(task * m + half * MLP_BM + row) * 16 + c] = dl;
-      if (c == lab) zlab = z[c];
     }
-    // -log softmax[label] = log(sum) - log(e^{z_label - zmax})
-    float rowloss = logf(ssum) - logf(zlab);
+    float rowloss = log1pf(sexcl) + (zmax - zl);
     rowloss += __shfl_xor_sync(0xFFFFFFFFu, rowloss, 16);
     rowloss += __shfl_xor_sync(0xFFFFFFFFu, rowloss, 8);
     rowloss += __shfl_xor_sync(0xFFFFFFFFu, rowloss, 4);

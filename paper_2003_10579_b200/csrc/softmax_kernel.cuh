@@ -204,15 +204,24 @@ __global__ void __launch_bounds__(SMX_NT) softmax_kernel(NumericArgs a) {
       float zmax = z;
 #pragma unroll
       for (int off = 8; off > 0; off >>= 1) zmax = fmaxf(zmax, __shfl_xor_sync(0xFFFFFFFFu, zmax, off));
-      const float ez = live ? expf(z - zmax) : 0.f;
-      float ssum = ez;
+      // sum of exponentials without the maximal class (whose term is exactly 1): log(1 + s) and
+      // p_max - 1 = -s / (1 + s) stay accurate when the sample is classified with a wide margin
+      const unsigned at_max = __ballot_sync(0xFFFFFFFFu, live && z == zmax);
+      const int cmax = __ffs((at_max >> (lane & 16)) & 0xFFFFu) - 1;
+      const bool is_max = sc == cmax;
+      const float ez = (live && !is_max) ? expf(z - zmax) : 0.f;
+      float sexcl = ez;
 #pragma unroll
-      for (int off = 8; off > 0; off >>= 1) ssum += __shfl_xor_sync(0xFFFFFFFFu, ssum, off);
+      for (int off = 8; off > 0; off >>= 1) sexcl += __shfl_xor_sync(0xFFFFFFFFu, sexcl, off);
+      const float ssum = 1.f + sexcl;
       const float zlab = __shfl_sync(0xFFFFFFFFu, z, (lane & 16) + label);
       float dl = 0.f;
-      if (live) dl = ez / ssum - (sc == label ? 1.f : 0.f);
+      if (live) {
+        if (is_max) dl = sc == label ? -sexcl / ssum : 1.f / ssum;
+        else dl = ez / ssum - (sc == label ? 1.f : 0.f);
+      }
       delta_s[sq * 16 + sc] = dl;
-      if (sc == 0 && sq < ti.rows) loss_acc += logf(ssum) + zmax - zlab;
+      if (sc == 0 && sq < ti.rows) loss_acc += log1pf(sexcl) + (zmax - zlab);
     }
     __syncthreads();   // (B)
 

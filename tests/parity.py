@@ -57,11 +57,26 @@ def assert_params_close(w_gpu, w_ora, what="", rtol=PARAM_RTOL):
     return e
 
 
-def assert_loss_close(l_gpu, l_ora, what="", rtol=LOSS_RTOL):
-    """Per update: |dL| <= rtol * max(|L_oracle|, 1e-6 * L_0), L_0 the first update's loss."""
+def assert_loss_close(l_gpu, l_ora, what="", rtol=LOSS_RTOL, gnorm=None, dw=0.0):
+    """Per update: |dL| <= rtol * max(|L_oracle|, 1e-6 * L_0) + 2 |g_j| dw.
+
+    L_0 is the first update's loss.  The second term is the first-order effect on the minibatch
+    loss of the parameter difference actually measured between the two trajectories (dw = the
+    largest |w_gpu - w_oracle|_2 seen at the compared steps, itself held to 1e-5 |w|; g_j = the
+    oracle's averaged gradient of update j, the gradient of that minibatch loss): two fp32-stored
+    trajectories drift apart by a few ulp per parameter, and a loss that has decayed by orders of
+    magnitude (or sits at its noise floor) magnifies that drift beyond any fixed relative bound.
+    Without gnorm the plain relative bound applies."""
     l_gpu, l_ora = np.asarray(l_gpu, np.float64), np.asarray(l_ora, np.float64)
     floor = 1e-6 * abs(l_ora.flat[0])
-    err = np.abs(l_gpu - l_ora) / np.maximum(np.abs(l_ora), floor)
-    assert err.max() <= rtol, "%s: loss relative error %.3g at update %d (gpu %.9g oracle %.9g)" % (
-        what, err.max(), int(err.argmax()), l_gpu.flat[err.argmax()], l_ora.flat[err.argmax()])
-    return err.max()
+    allow = rtol * np.maximum(np.abs(l_ora), floor)
+    if gnorm is not None:
+        allow = allow + 2.0 * np.asarray(gnorm, np.float64) * dw
+    err = np.abs(l_gpu - l_ora)
+    bad = err > allow
+    if bad.any():
+        j = int(np.argmax(err / allow))
+        raise AssertionError("%s: loss differs by %.3g (allowed %.3g) at update %d (gpu %.9g oracle %.9g)" % (
+            what, err.flat[j], allow.flat[j], j, l_gpu.flat[j], l_ora.flat[j]))
+    rel = err / np.maximum(np.abs(l_ora), floor)
+    return rel.max()
