@@ -51,7 +51,7 @@ def _load():
                              i64, vp, C.POINTER(vp)]
     L.sim_set_params.argtypes = [vp, vp]
     L.sim_set_adasync.argtypes = [vp, i32, dbl]
-    L.sim_set_tuning.argtypes = [vp, i32]
+    L.sim_set_tuning.argtypes = [vp, i32, i32, i32]
     L.sim_reserve.argtypes = [vp, i64]
     L.sim_run.argtypes = [vp, i64]
     L.sim_trace_size.argtypes = [vp, C.POINTER(i64), C.POINTER(i32)]
@@ -138,8 +138,8 @@ class Simulation:
     def set_adasync(self, K0, t_interval):
         _check(lib.sim_set_adasync(self._h, K0, t_interval), self._h)
 
-    def set_tuning(self, stages=0):
-        _check(lib.sim_set_tuning(self._h, stages), self._h)
+    def set_tuning(self, stages=0, tile_rows=0, threads=0):
+        _check(lib.sim_set_tuning(self._h, stages, tile_rows, threads), self._h)
 
     def reserve(self, total_updates):
         _check(lib.sim_reserve(self._h, total_updates), self._h)

@@ -50,7 +50,7 @@ struct sim_handle {
   int n_slots = 0;
   long long n_params = 0;
   long long n_updates = 0, cap = 0;
-  int tune_stages = 0;
+  int tune_stages = 0, tune_rows = 0, tune_threads = 0;
   // device state
   uint32_t* s = nullptr;
   uint32_t* tau = nullptr;
@@ -168,7 +168,8 @@ sim_status launch_linear1(sim_handle* h, NumericArgs& a) {
   const size_t row_bytes = (size_t)d * 4;
   int S = h->tune_stages;
   if (S <= 0) {
-    const size_t budget = d <= 1024 ? (36u << 10) : (200u << 10);
+    // small rows: several CTAs per SM; long rows: one CTA per SM, or two when there are more replicas than SMs
+    const size_t budget = d <= 1024 ? (36u << 10) : (a.R > 148 ? (100u << 10) : (200u << 10));
     S = (int)(budget / ((size_t)T * row_bytes));
   }
   if (S < 2) S = 2;
@@ -191,7 +192,11 @@ sim_status run_linear1(sim_handle* h, NumericArgs& a) {
   if (d4 <= 128) return launch_linear1<128, 1, 4>(h, a);
   if (d4 <= 256) return launch_linear1<128, 2, 4>(h, a);
   if (d4 <= 512) return launch_linear1<256, 2, 4>(h, a);
-  if (d4 <= 1024) return launch_linear1<256, 4, 4>(h, a);
+  if (d4 <= 1024) {
+    const int rows = h->tune_rows ? h->tune_rows : (a.R > 148 ? 2 : 4), threads = h->tune_threads ? h->tune_threads : 256;
+    if (threads == 512 && d4 <= 1024) return rows == 2 ? launch_linear1<512, 2, 2>(h, a) : launch_linear1<512, 2, 4>(h, a);
+    return rows == 2 ? launch_linear1<256, 4, 2>(h, a) : launch_linear1<256, 4, 4>(h, a);
+  }
   if (d4 <= 2048) return launch_linear1<512, 4, 2>(h, a);
   return fail(h, SIM_ERR_ARG, "d > 8192 is not supported by the linear-model kernel");
 }
@@ -324,10 +329,12 @@ sim_status sim_set_adasync(sim_handle* h, int32_t K0, double t_interval) {
   return SIM_OK;
 }
 
-sim_status sim_set_tuning(sim_handle* h, int32_t stages) {
+sim_status sim_set_tuning(sim_handle* h, int32_t stages, int32_t tile_rows, int32_t threads) {
   if (!h) return fail(nullptr, SIM_ERR_ARG, "handle is NULL");
   if (stages < 0 || stages == 1 || stages > 8) return fail(h, SIM_ERR_ARG, "stages must be 0 (automatic) or in [2, 8]");
-  h->tune_stages = stages;
+  if (tile_rows != 0 && tile_rows != 2 && tile_rows != 4) return fail(h, SIM_ERR_ARG, "tile_rows must be 0, 2 or 4");
+  if (threads != 0 && threads != 256 && threads != 512) return fail(h, SIM_ERR_ARG, "threads must be 0, 256 or 512");
+  h->tune_stages = stages; h->tune_rows = tile_rows; h->tune_threads = threads;
   return SIM_OK;
 }
 
