@@ -9,14 +9,14 @@
 // everything else (bias, relu, layer 2, softmax, loss, update) is fp32.
 //
 // All replicas advance in lock step, one update at a time, with four launches per update:
-//   forward   one CTA per (replica, contributor, 64-sample half): A1 tile 64 x H by mma.sync
-//             m16n8k16 (cp.async 3-stage ring, XOR-swizzled shared memory, ldmatrix), then
-//             h = relu(A1 + b1), logits, softmax, delta2, delta1 = (delta2 W2^T) . [h > 0];
-//             writes h, delta2, bf16(delta1), partial db1 and the loss of its rows
+//   forward   (mlp_tc_kernel.cuh) one CTA per (replica, contributor, 128-sample block): A1 = X_b W1 on
+//             tcgen05 with the accumulator in tensor memory, then h = relu(A1 + b1), logits, softmax,
+//             delta2, delta1 = (delta2 W2^T) . [h > 0]; writes h, delta2, bf16(delta1), partial db1, loss
 //   head      one CTA per (replica, contributor): dW2 = h^T delta2, db2
 //   dw1       one CTA per (replica, 64-row slab of W1): accumulates X^T delta1 over all K m samples
-//             of the update in registers and applies W1 <- W1 - (eta/(K m)) dW1 in its epilogue
-//             (Eq. 2 / Eq. 3), writing the new version and its bf16 shadow: dW1 never exists in memory
+//             of the update (mma.sync m16n8k16, cp.async 3-stage ring, XOR-swizzled shared memory,
+//             ldmatrix) and applies W1 <- W1 - (eta/(K m)) dW1 in its epilogue (Eq. 2 / Eq. 3), writing
+//             the new version and its transposed bf16 shadow: dW1 never exists in memory
 //   small     b1, W2, b2 update from the partials (fixed summation order), loss record
 #pragma once
 #include <cuda_bf16.h>
@@ -27,14 +27,14 @@ namespace ssim {
 
 struct MlpScratch {
   __nv_bfloat16* Xq = nullptr;     // [n][d]                   bf16 copy of the data set
-  __nv_bfloat16* W1q = nullptr;    // [R][n_slots][d*H]        bf16 shadow of every W1 version
+  __nv_bfloat16* W1qT = nullptr;   // [R][n_slots][H][d]       bf16 shadow of every W1 version, transposed (d contiguous)
   __nv_bfloat16* D1q = nullptr;    // [R][Kmax][m][H]          bf16(delta1) of the current update
   float* Hact = nullptr;           // [R][Kmax][m][H]          h
   float* D2 = nullptr;             // [R][Kmax][m][16]         delta2
-  float* db1_part = nullptr;       // [R][Kmax][m/64][H]
+  float* db1_part = nullptr;       // [R][Kmax][m/32][H]       column sums of delta1 per 32-row group
   float* dW2_part = nullptr;       // [R][Kmax][H*C]
   float* db2_part = nullptr;       // [R][Kmax][16]
-  float* loss_part = nullptr;      // [R][Kmax][m/64]
+  float* loss_part = nullptr;      // [R][Kmax][m/32]
   int H = 0, C = 0, d = 0, m = 0, Kmax = 0, n_slots = 0, R = 0;
   long long n = 0;
 };
@@ -57,7 +57,7 @@ constexpr int MLP_SMEM = MLP_STAGES * (MLP_STAGE_A + MLP_STAGE_B) + 1024;
 inline const char* mlp_shape_unsupported(int d, int H, int C, int m) {
   if (H < 64 || H > 512 || H % 64 != 0) return "mlp: hidden width must be a multiple of 64 in [64, 512]";
   if (d % 64 != 0) return "mlp: d must be a multiple of 64";
-  if (m % 64 != 0) return "mlp: m must be a multiple of 64";
+  if (m % 128 != 0) return "mlp: m must be a multiple of 128";
   if (C < 2 || C > 16) return "mlp: n_classes must be in [2, 16]";
   return nullptr;
 }
@@ -138,258 +138,13 @@ __global__ void to_bf16_kernel(const float* src, __nv_bfloat16* dst, long long c
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < count; i += (long long)gridDim.x * blockDim.x)
     dst[i] = __float2bfloat16_rn(src[i]);
 }
-// bf16 shadow of W1 of pool slot `slot` of every replica
-__global__ void shadow_w1_kernel(const float* pool, __nv_bfloat16* W1q, long long n_params, long long dH, int n_slots, int slot, int R) {
-  const long long total = dH * R;
+// transposed bf16 shadow (W1^T [H][d]) of W1 in pool slot `slot` of every replica
+__global__ void shadow_w1_kernel(const float* pool, __nv_bfloat16* W1qT, long long n_params, int d, int H, int n_slots, int slot, int R) {
+  const long long dH = (long long)d * H, total = dH * R;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
     const long long r = i / dH, p = i % dH;
-    W1q[((size_t)r * n_slots + slot) * dH + p] = __float2bfloat16_rn(pool[((size_t)r * n_slots + slot) * n_params + p]);
-  }
-}
-
-// ---- forward + backward down to delta1 -------------------------------------------------------
-__global__ void __launch_bounds__(256, 1) mlp_forward_kernel(MlpArgs g) {
-  const NumericArgs& a = g.na;
-  const MlpScratch& sc = g.sc;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int H = sc.H, C = sc.C, d = sc.d, m = sc.m;
-  const int halves = m / MLP_BM;
-  const int half = blockIdx.x % halves;
-  const int l = (blockIdx.x / halves) % sc.Kmax;
-  const int r = blockIdx.x / (halves * sc.Kmax);
-  const long long j = g.j;
-  const int K = (int)a.K_used[(size_t)r * a.cap + j];
-  if (l >= K) return;
-  const size_t ent = ((size_t)r * a.cap + j) * a.K_stride + l;
-  const uint32_t worker = a.worker[ent], seq = a.seq[ent];
-  const int snap = mlp_snap_slot(a, r, j, l);
-  const uint32_t rid = a.replica_base + (uint32_t)r;
-  const size_t task = (size_t)r * sc.Kmax + l;
-  const long long dH = (long long)d * H;
-  const float* wsnap = a.pool + ((size_t)r * a.n_slots + snap) * a.n_params;
-  const __nv_bfloat16* W1q = sc.W1q + ((size_t)r * sc.n_slots + snap) * dH;
-
-  extern __shared__ __align__(128) unsigned char smem[];
-  unsigned long long* rowptr_s = reinterpret_cast<unsigned long long*>(smem);   // [64] source rows (element offsets)
-  int* label_s = reinterpret_cast<int*>(smem + 512);                            // [64]
-  unsigned char* stages = smem + 1024;
-  const uint32_t stages_addr = smem_addr(stages);
-
-  if (tid < MLP_BM) {
-    uint32_t idx = draw_index(a.seed, rid, worker, seq, (uint32_t)(half * MLP_BM + tid), a.n);
-    if ((uint64_t)idx >= a.n) { atomicExch(a.err, ERR_BAD_INDEX); idx = 0; }
-    rowptr_s[tid] = (unsigned long long)idx * (unsigned long long)d;
-    label_s[tid] = reinterpret_cast<const int*>(a.y)[idx];
-  }
-  __syncthreads();
-
-  auto load_stage = [&](int kc) {
-    const int st = kc % MLP_STAGES;
-    const uint32_t As = stages_addr + st * (MLP_STAGE_A + MLP_STAGE_B);
-    const uint32_t Bs = As + MLP_STAGE_A;
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      const int c = tid + 256 * i, row = c >> 3, ch = c & 7;
-      cp_async16(As + row * 128 + ((ch ^ (row & 7)) << 4), sc.Xq + rowptr_s[row] + (size_t)kc * MLP_BK + ch * 8);
-    }
-    const int nch = H / 8;   // 16-byte chunks per k-row
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const int c = tid + 256 * i, krow = c >> 6, ch = c & 63;
-      if (ch < nch)
-        cp_async16(Bs + krow * MLP_PITCH_B + ((ch ^ (krow & 7)) << 4), W1q + ((size_t)kc * MLP_BK + krow) * H + ch * 8);
-    }
-  };
-
-  float acc[4][8][4];
-#pragma unroll
-  for (int mt = 0; mt < 4; ++mt)
-#pragma unroll
-    for (int nt = 0; nt < 8; ++nt)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) acc[mt][nt][e] = 0.f;
-
-  const int nk = d / MLP_BK;
-  for (int s = 0; s < MLP_STAGES - 1; ++s) { if (s < nk) load_stage(s); cp_async_commit(); }
-  for (int kc = 0; kc < nk; ++kc) {
-    cp_async_wait<MLP_STAGES - 2>();
-    __syncthreads();
-    if (kc + MLP_STAGES - 1 < nk) load_stage(kc + MLP_STAGES - 1);
-    cp_async_commit();
-    const int st = kc % MLP_STAGES;
-    const uint32_t As = stages_addr + st * (MLP_STAGE_A + MLP_STAGE_B);
-    mlp_tile_mma<false>(acc, As, As + MLP_STAGE_A, warp, lane, H);
-  }
-  cp_async_wait<0>();
-  __syncthreads();
-
-  // ---- epilogue: the stage buffers are free; reuse them ----
-  float* W2_s = reinterpret_cast<float*>(stages);                 // [H][16]
-  float* zpart_s = W2_s + 512 * 16;                                // [8 warps][64 rows][16]
-  float* d2_s = zpart_s + 8 * 64 * 16;                             // [64][16]
-  const float* b1 = wsnap + dH;
-  const float* W2 = b1 + H;
-  const float* b2 = W2 + (size_t)H * C;
-  for (int i = tid; i < H * 16; i += 256) {
-    const int col = i >> 4, c = i & 15;
-    W2_s[i] = c < C ? W2[(size_t)col * C + c] : 0.f;
-  }
-  const int g8 = lane >> 2, tig = lane & 3;
-  const bool wactive = warp * 64 < H;
-  // h = relu(A1 + b1); keep in acc; write to the scratch for the head kernel
-  if (wactive) {
-#pragma unroll
-    for (int nt = 0; nt < 8; ++nt) {
-      const int col = warp * 64 + nt * 8 + 2 * tig;
-      const float bb0 = b1[col], bb1 = b1[col + 1];
-#pragma unroll
-      for (int mt = 0; mt < 4; ++mt) {
-#pragma unroll
-        for (int rh = 0; rh < 2; ++rh) {
-          const int row = mt * 16 + g8 + rh * 8;
-          const float h0 = fmaxf(acc[mt][nt][2 * rh] + bb0, 0.f), h1 = fmaxf(acc[mt][nt][2 * rh + 1] + bb1, 0.f);
-          acc[mt][nt][2 * rh] = h0; acc[mt][nt][2 * rh + 1] = h1;
-          *reinterpret_cast<float2*>(sc.Hact + (task * m + half * MLP_BM + row) * H + col) = make_float2(h0, h1);
-        }
-      }
-    }
-  }
-  __syncthreads();   // W2_s ready
-  // partial logits over this warp's 64 hidden units
-#pragma unroll
-  for (int mt = 0; mt < 4; ++mt) {
-#pragma unroll
-    for (int rh = 0; rh < 2; ++rh) {
-      const int row = mt * 16 + g8 + rh * 8;
-      float zp[16];
-#pragma unroll
-      for (int c = 0; c < 16; ++c) zp[c] = 0.f;
-      if (wactive) {
-#pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
-#pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const int col = warp * 64 + nt * 8 + 2 * tig + e;
-            const float hv = acc[mt][nt][2 * rh + e];
-            const float4* wr = reinterpret_cast<const float4*>(W2_s + col * 16);
-#pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4) {
-              const float4 w = wr[c4];
-              zp[4 * c4] = fmaf(hv, w.x, zp[4 * c4]); zp[4 * c4 + 1] = fmaf(hv, w.y, zp[4 * c4 + 1]);
-              zp[4 * c4 + 2] = fmaf(hv, w.z, zp[4 * c4 + 2]); zp[4 * c4 + 3] = fmaf(hv, w.w, zp[4 * c4 + 3]);
-            }
-          }
-        }
-      }
-#pragma unroll
-      for (int c = 0; c < 16; ++c) {
-        zp[c] += __shfl_xor_sync(0xFFFFFFFFu, zp[c], 1);
-        zp[c] += __shfl_xor_sync(0xFFFFFFFFu, zp[c], 2);
-      }
-      if (tig == 0) {
-#pragma unroll
-        for (int c4 = 0; c4 < 4; ++c4)
-          reinterpret_cast<float4*>(zpart_s + (warp * 64 + row) * 16)[c4] = make_float4(zp[4 * c4], zp[4 * c4 + 1], zp[4 * c4 + 2], zp[4 * c4 + 3]);
-      }
-    }
-  }
-  __syncthreads();
-  // softmax, loss and delta2: one thread per row
-  if (tid < MLP_BM) {
-    const int row = tid, lab = label_s[row];
-    float z[16], zmax = -INFINITY;
-#pragma unroll
-    for (int c = 0; c < 16; ++c) {
-      float s = 0.f;
-      for (int w = 0; w < 8; ++w) s += zpart_s[(w * 64 + row) * 16 + c];
-      z[c] = c < C ? s + b2[c] : -INFINITY;
-      zmax = fmaxf(zmax, z[c]);
-    }
-    // exponentials without the maximal class (its term is exactly 1): log(1 + s) and
-    // p_max - 1 = -s / (1 + s) stay accurate for samples classified with a wide margin
-    int cmax = 0;
-#pragma unroll
-    for (int c = 15; c >= 0; --c) if (c < C && z[c] == zmax) cmax = c;
-    float zl = 0.f;
-#pragma unroll
-    for (int c = 0; c < 16; ++c) if (c == lab) zl = z[c];
-    float sexcl = 0.f;
-#pragma unroll
-    for (int c = 0; c < 16; ++c) { z[c] = (c < C && c != cmax) ? expf(z[c] - zmax) : 0.f; sexcl += z[c]; }
-    const float ssum = 1.f + sexcl;
-#pragma unroll
-    for (int c = 0; c < 16; ++c) {
-      float dl = 0.f;
-      if (c < C) {
-        if (c == cmax) dl = c == lab ? -sexcl / ssum : 1.f / ssum;
-        else dl = z[c] / ssum - (c == lab ? 1.f : 0.f);
-      }
-      d2_s[row * 16 + c] = dl;
-      sc.D2[(task * m + half * MLP_BM + row) * 16 + c] = dl;
-    }
-    float rowloss = log1pf(sexcl) + (zmax - zl);
-    rowloss += __shfl_xor_sync(0xFFFFFFFFu, rowloss, 16);
-    rowloss += __shfl_xor_sync(0xFFFFFFFFu, rowloss, 8);
-    rowloss += __shfl_xor_sync(0xFFFFFFFFu, rowloss, 4);
-    rowloss += __shfl_xor_sync(0xFFFFFFFFu, rowloss, 2);
-    rowloss += __shfl_xor_sync(0xFFFFFFFFu, rowloss, 1);
-    if (lane == 0) d2_s[MLP_BM * 16 + warp] = rowloss;     // rows 0..31 and rows 32..63
-  }
-  __syncthreads();
-  if (tid == 0) sc.loss_part[task * halves + half] = d2_s[MLP_BM * 16] + d2_s[MLP_BM * 16 + 1];
-  // delta1 = (delta2 W2^T) . [h > 0]; db1 partial; bf16 store
-  if (wactive) {
-#pragma unroll
-    for (int nt = 0; nt < 8; ++nt) {
-      float colsum[2] = {0.f, 0.f};
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int col = warp * 64 + nt * 8 + 2 * tig + e;
-        float w2[16];
-#pragma unroll
-        for (int c4 = 0; c4 < 4; ++c4) {
-          const float4 w = reinterpret_cast<const float4*>(W2_s + col * 16)[c4];
-          w2[4 * c4] = w.x; w2[4 * c4 + 1] = w.y; w2[4 * c4 + 2] = w.z; w2[4 * c4 + 3] = w.w;
-        }
-#pragma unroll
-        for (int mt = 0; mt < 4; ++mt) {
-#pragma unroll
-          for (int rh = 0; rh < 2; ++rh) {
-            const int row = mt * 16 + g8 + rh * 8;
-            float dv = 0.f;
-#pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4) {
-              const float4 dl = reinterpret_cast<const float4*>(d2_s + row * 16)[c4];
-              dv = fmaf(dl.x, w2[4 * c4], dv); dv = fmaf(dl.y, w2[4 * c4 + 1], dv);
-              dv = fmaf(dl.z, w2[4 * c4 + 2], dv); dv = fmaf(dl.w, w2[4 * c4 + 3], dv);
-            }
-            dv = acc[mt][nt][2 * rh + e] > 0.f ? dv : 0.f;
-            acc[mt][nt][2 * rh + e] = dv;
-            colsum[e] += dv;
-          }
-        }
-      }
-      const int col = warp * 64 + nt * 8 + 2 * tig;
-#pragma unroll
-      for (int mt = 0; mt < 4; ++mt) {
-#pragma unroll
-        for (int rh = 0; rh < 2; ++rh) {
-          const int row = mt * 16 + g8 + rh * 8;
-          *reinterpret_cast<__nv_bfloat162*>(sc.D1q + (task * m + half * MLP_BM + row) * H + col) =
-              __floats2bfloat162_rn(acc[mt][nt][2 * rh], acc[mt][nt][2 * rh + 1]);
-        }
-      }
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        colsum[e] += __shfl_xor_sync(0xFFFFFFFFu, colsum[e], 4);
-        colsum[e] += __shfl_xor_sync(0xFFFFFFFFu, colsum[e], 8);
-        colsum[e] += __shfl_xor_sync(0xFFFFFFFFu, colsum[e], 16);
-      }
-      if (g8 == 0) {
-        sc.db1_part[(task * halves + half) * H + col] = colsum[0];
-        sc.db1_part[(task * halves + half) * H + col + 1] = colsum[1];
-      }
-    }
+    const long long n = p / d, k = p % d;       // output element (n, k) = W1[k][n]
+    W1qT[((size_t)r * n_slots + slot) * dH + p] = __float2bfloat16_rn(pool[((size_t)r * n_slots + slot) * n_params + k * H + n]);
   }
 }
 
@@ -511,7 +266,7 @@ __global__ void __launch_bounds__(256, 1) mlp_dw1_update_kernel(MlpArgs g) {
   const float scale = (float)((double)a.eta / ((double)K * (double)m));
   const float* wc = a.pool + ((size_t)r * a.n_slots + cur) * a.n_params;
   float* wn = a.pool + ((size_t)r * a.n_slots + fresh) * a.n_params;
-  __nv_bfloat16* wq = sc.W1q + ((size_t)r * sc.n_slots + fresh) * dH;
+  __nv_bfloat16* wq = sc.W1qT + ((size_t)r * sc.n_slots + fresh) * dH;   // [H][d]
   const int g8 = lane >> 2, tig = lane & 3;
 #pragma unroll
   for (int mt = 0; mt < 4; ++mt) {
@@ -524,7 +279,8 @@ __global__ void __launch_bounds__(256, 1) mlp_dw1_update_kernel(MlpArgs g) {
         const float2 w = *reinterpret_cast<const float2*>(wc + row * H + col);
         const float n0 = fmaf(-scale, acc[mt][nt][2 * rh], w.x), n1 = fmaf(-scale, acc[mt][nt][2 * rh + 1], w.y);
         *reinterpret_cast<float2*>(wn + row * H + col) = make_float2(n0, n1);
-        *reinterpret_cast<__nv_bfloat162*>(wq + row * H + col) = __floats2bfloat162_rn(n0, n1);
+        wq[(size_t)col * d + row] = __float2bfloat16_rn(n0);
+        wq[(size_t)(col + 1) * d + row] = __float2bfloat16_rn(n1);
       }
     }
   }
@@ -537,7 +293,7 @@ __global__ void __launch_bounds__(256) mlp_small_update_kernel(MlpArgs g) {
   const int r = blockIdx.x, tid = threadIdx.x;
   const long long j = g.j;
   const int K = (int)a.K_used[(size_t)r * a.cap + j];
-  const int H = sc.H, C = sc.C, m = sc.m, halves = m / MLP_BM;
+  const int H = sc.H, C = sc.C, m = sc.m, halves = m / 32;   // partial sums per 32-row group
   const long long dH = (long long)sc.d * H;
   const int cur = mlp_cur_slot(a, r, j), fresh = mlp_fresh_slot(a, r, j);
   const float scale = (float)((double)a.eta / ((double)K * (double)m));
@@ -565,7 +321,7 @@ __global__ void __launch_bounds__(256) mlp_small_update_kernel(MlpArgs g) {
 
 // ---- host side -----------------------------------------------------------------------------------
 inline void mlp_scratch_free(MlpScratch& s) {
-  cudaFree(s.Xq); cudaFree(s.W1q); cudaFree(s.D1q); cudaFree(s.Hact); cudaFree(s.D2);
+  cudaFree(s.Xq); cudaFree(s.W1qT); cudaFree(s.D1q); cudaFree(s.Hact); cudaFree(s.D2);
   cudaFree(s.db1_part); cudaFree(s.dW2_part); cudaFree(s.db2_part); cudaFree(s.loss_part);
   s = MlpScratch{};
 }
@@ -579,14 +335,14 @@ inline cudaError_t mlp_scratch_alloc(MlpScratch& s, const float* X, long long n,
   if ((e = cudaMalloc(reinterpret_cast<void**>(&(ptr)), (count) * sizeof(*(ptr)))) != cudaSuccess) return e; \
   if ((e = cudaMemsetAsync((ptr), 0, (count) * sizeof(*(ptr)), stream)) != cudaSuccess) return e;
   MLP_ALLOC(s.Xq, (size_t)n * d)
-  MLP_ALLOC(s.W1q, (size_t)R * n_slots * d * H)
+  MLP_ALLOC(s.W1qT, (size_t)R * n_slots * d * H)
   MLP_ALLOC(s.D1q, tasks * m * H)
   MLP_ALLOC(s.Hact, tasks * m * H)
   MLP_ALLOC(s.D2, tasks * m * 16)
-  MLP_ALLOC(s.db1_part, tasks * (m / MLP_BM) * H)
+  MLP_ALLOC(s.db1_part, tasks * (m / 32) * H)
   MLP_ALLOC(s.dW2_part, tasks * H * C)
   MLP_ALLOC(s.db2_part, tasks * 16)
-  MLP_ALLOC(s.loss_part, tasks * (m / MLP_BM))
+  MLP_ALLOC(s.loss_part, tasks * (m / 32))
 #undef MLP_ALLOC
   to_bf16_kernel<<<1184, 256, 0, stream>>>(X, s.Xq, (long long)n * d);
   return cudaGetLastError();
@@ -594,27 +350,8 @@ inline cudaError_t mlp_scratch_alloc(MlpScratch& s, const float* X, long long n,
 
 // after the initial parameters went into slot 0 of every replica
 inline cudaError_t mlp_after_set_params(MlpScratch& s, const float* pool, long long n_params, cudaStream_t stream) {
-  shadow_w1_kernel<<<1184, 256, 0, stream>>>(pool, s.W1q, n_params, (long long)s.d * s.H, s.n_slots, 0, s.R);
+  shadow_w1_kernel<<<1184, 256, 0, stream>>>(pool, s.W1qT, n_params, s.d, s.H, s.n_slots, 0, s.R);
   return cudaGetLastError();
-}
-
-inline cudaError_t run_mlp(NumericArgs& a, MlpScratch& s, int P, cudaStream_t stream, const char** why) {
-  *why = nullptr;
-  cudaError_t e;
-  if ((e = cudaFuncSetAttribute(mlp_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MLP_SMEM)) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(mlp_dw1_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MLP_SMEM + 1024)) != cudaSuccess) return e;
-  MlpArgs g{};
-  g.na = a; g.sc = s; g.H = s.H; g.P = P;
-  const int halves = s.m / MLP_BM;
-  for (long long u = 0; u < a.iters; ++u) {
-    g.j = a.j0 + u;
-    mlp_forward_kernel<<<a.R * s.Kmax * halves, 256, MLP_SMEM, stream>>>(g);
-    mlp_head_kernel<<<a.R * s.Kmax, 512, (size_t)s.m * 16 * 4, stream>>>(g);
-    mlp_dw1_update_kernel<<<a.R * (s.d / MLP_BM), 256, MLP_SMEM + 1024, stream>>>(g);
-    mlp_small_update_kernel<<<a.R, 256, 0, stream>>>(g);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
-  }
-  return cudaSuccess;
 }
 
 }  // namespace ssim

@@ -1,0 +1,376 @@
+// MLP forward pass on the 5th-generation tensor cores (tcgen05) with the accumulator in tensor
+// memory.
+//
+// One CTA per (replica, contributor, 128-sample block):  A1[128 x H] = bf16(X_b)[128 x d] bf16(W1)[d x H]
+//   warp 0   producer: TMA tensor loads into a ring of shared-memory stages (128-byte swizzle);
+//            the 128 gathered sample rows go in as 128 one-row boxes of 64 features, the W1 tile
+//            comes from the transposed bf16 shadow W1^T [H][d] (K-major B operand) as one or two boxes
+//   warp 1   allocates tensor memory; one elected lane issues tcgen05.mma (M=128, N<=256, K=16)
+//            and commits stage-free / accumulator-ready mbarriers
+//   warps 2-5  epilogue: tcgen05.ld gives each thread one sample's full row of A1, so bias, relu,
+//            the 10-way head, softmax and delta2 need no cross-thread reduction; a second pass
+//            over tensor memory forms delta1 = (delta2 W2^T) . [A1 + b1 > 0], stores it in bf16
+//            and reduces its column sums (db1) with a warp transposition reduce
+// Every mbarrier wait is bounded; a wait that runs out sets the error word and the CTA drains.
+#pragma once
+#include <cuda.h>
+
+#include "mlp_kernel.cuh"
+#include "softmax_kernel.cuh"
+
+namespace ssim {
+
+constexpr int TC_BK = 64;                       // k per stage: one 128-byte swizzle atom of bf16
+constexpr int TC_A_BYTES = 128 * 128;           // 128 rows x 128 B
+constexpr int TC_THREADS = 192;
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_alloc(uint32_t smem_dst, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tc_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]),
+        "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]),
+        "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]),
+        "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  K-major operand: rows (M or N) are 128 B
+// apart, 8-row groups 1024 B apart (stride byte offset); the leading byte offset is unused.
+__device__ __forceinline__ uint64_t tc_desc_kmajor(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
+         ((uint64_t)2 << 61);
+}
+// bf16 x bf16 -> f32, M = 128, N = n, both operands K-major
+__device__ __forceinline__ uint32_t tc_idesc(int n, int a_mn_major, int b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
+         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+struct TcLayout {   // shared-memory plan of the forward kernel (offsets from a 1024-byte aligned base)
+  int stages, stage_bytes, off_w2, off_b1, off_b2, off_rows, off_labels, off_bars, off_tmem, total;
+};
+inline __host__ __device__ TcLayout tc_forward_layout(int H) {
+  TcLayout L;
+  L.stage_bytes = TC_A_BYTES + H * 128;
+  L.stages = H <= 256 ? 4 : 2;
+  L.off_w2 = L.stages * L.stage_bytes;
+  L.off_b1 = L.off_w2 + H * 16 * 4;
+  L.off_b2 = L.off_b1 + H * 4;
+  L.off_rows = L.off_b2 + 64;
+  L.off_labels = L.off_rows + 128 * 4;
+  L.off_bars = L.off_labels + 128 * 4;
+  L.off_tmem = L.off_bars + 8 * (2 * L.stages + 1);
+  L.total = L.off_tmem + 16 + 1024;   // slack for the manual 1024-byte alignment
+  return L;
+}
+
+__global__ void __launch_bounds__(TC_THREADS, 1)
+mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, MlpArgs g) {
+  const NumericArgs& a = g.na;
+  const MlpScratch& sc = g.sc;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int H = sc.H, C = sc.C, d = sc.d, m = sc.m;
+  const int mtiles = m / 128;
+  const int mt = blockIdx.x % mtiles;
+  const int l = (blockIdx.x / mtiles) % sc.Kmax;
+  const int r = blockIdx.x / (mtiles * sc.Kmax);
+  const long long j = g.j;
+  const int K = (int)a.K_used[(size_t)r * a.cap + j];
+  if (l >= K) return;
+  const size_t ent = ((size_t)r * a.cap + j) * a.K_stride + l;
+  const uint32_t worker = a.worker[ent], seq = a.seq[ent];
+  const int snap = mlp_snap_slot(a, r, j, l);
+  const uint32_t rid = a.replica_base + (uint32_t)r;
+  const size_t task = (size_t)r * sc.Kmax + l;
+  const long long dH = (long long)d * H;
+  const float* wsnap = a.pool + ((size_t)r * a.n_slots + snap) * a.n_params;
+  const int n_halves = H > 256 ? 2 : 1;
+  const int n_inst = H / n_halves;
+  uint32_t tmem_cols = 32;
+  while ((int)tmem_cols < H) tmem_cols <<= 1;
+
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw_addr = smem_addr(smem_raw);
+  const uint32_t base_addr = (raw_addr + 1023u) & ~1023u;
+  unsigned char* base = smem_raw + (base_addr - raw_addr);
+  const TcLayout L = tc_forward_layout(H);
+  const int S = L.stages;
+  float* W2_s = reinterpret_cast<float*>(base + L.off_w2);
+  float* b1_s = reinterpret_cast<float*>(base + L.off_b1);
+  float* b2_s = reinterpret_cast<float*>(base + L.off_b2);
+  int* rows_s = reinterpret_cast<int*>(base + L.off_rows);
+  int* label_s = reinterpret_cast<int*>(base + L.off_labels);
+  const uint32_t bars = base_addr + L.off_bars;            // full[S] | empty[S] | acc_ready
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base + L.off_tmem);
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (S + s); };
+  const uint32_t acc_bar = bars + 8u * (2 * S);
+
+  if (tid == 0) {
+    for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    mbar_init(acc_bar, 1);
+    mbar_fence_init();
+  }
+  if (warp == 1) tc_alloc(smem_addr(tmem_slot), tmem_cols);
+  {
+    const float* b1 = wsnap + dH;
+    const float* W2 = b1 + H;
+    const float* b2 = W2 + (size_t)H * C;
+    for (int i = tid; i < H * 16; i += TC_THREADS) {
+      const int col = i >> 4, c = i & 15;
+      W2_s[i] = c < C ? W2[(size_t)col * C + c] : 0.f;
+    }
+    for (int i = tid; i < H; i += TC_THREADS) b1_s[i] = b1[i];
+    if (tid < 16) b2_s[tid] = tid < C ? b2[tid] : 0.f;
+    if (tid < 128) {
+      uint32_t idx = draw_index(a.seed, rid, worker, seq, (uint32_t)(mt * 128 + tid), a.n);
+      if ((uint64_t)idx >= a.n) { atomicExch(a.err, ERR_BAD_INDEX); idx = 0; }
+      rows_s[tid] = (int)idx;
+      label_s[tid] = reinterpret_cast<const int*>(a.y)[idx];
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int nk = d / TC_BK;
+  bool failed = false;
+
+  if (warp == 0) {
+    // ---- producer ----
+    const int w_row0 = (int)(((size_t)r * sc.n_slots + snap) * H);
+    for (int kc = 0; kc < nk; ++kc) {
+      const int s = kc % S;
+      if (!mbar_wait(empty_bar(s), (uint32_t)(((kc / S) & 1) ^ 1))) { failed = true; break; }
+      const uint32_t As = base_addr + (uint32_t)s * L.stage_bytes, Bs = As + TC_A_BYTES;
+      if (lane == 0) {
+        mbar_arrive_expect_tx(full_bar(s), (uint32_t)L.stage_bytes);
+        for (int hf = 0; hf < n_halves; ++hf)
+          tma_load_2d(Bs + (uint32_t)hf * n_inst * 128, &tmW, kc * TC_BK, w_row0 + hf * n_inst, full_bar(s));
+      }
+      __syncwarp();
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int row = lane + 32 * i;
+        tma_load_2d(As + (uint32_t)row * 128, &tmX, kc * TC_BK, rows_s[row], full_bar(s));
+      }
+    }
+  } else if (warp == 1) {
+    // ---- MMA issuer ----
+    const uint32_t idesc = tc_idesc(n_inst, 0, 0);
+    for (int kc = 0; kc < nk; ++kc) {
+      const int s = kc % S;
+      if (!mbar_wait(full_bar(s), (uint32_t)((kc / S) & 1))) { failed = true; break; }
+      tc_fence_after();
+      if (lane == 0) {
+        const uint32_t As = base_addr + (uint32_t)s * L.stage_bytes, Bs = As + TC_A_BYTES;
+#pragma unroll
+        for (int k16 = 0; k16 < TC_BK / 16; ++k16) {
+          const uint64_t ad = tc_desc_kmajor(As + k16 * 32);
+          for (int hf = 0; hf < n_halves; ++hf) {
+            const uint64_t bd = tc_desc_kmajor(Bs + (uint32_t)hf * n_inst * 128 + k16 * 32);
+            tc_mma_bf16(tmem_base + (uint32_t)hf * n_inst, ad, bd, idesc, (kc > 0 || k16 > 0) ? 1u : 0u);
+          }
+        }
+        tc_commit(empty_bar(s));                    // the stage may be refilled once these MMAs have read it
+        if (kc == nk - 1) tc_commit(acc_bar);       // accumulator complete
+      }
+      __syncwarp();
+    }
+  } else {
+    // ---- epilogue: thread = one sample row ----
+    const int q = warp & 3;                         // the TMEM lane quarter this warp may read
+    const int row = 32 * q + lane;
+    const size_t grow = task * m + (size_t)mt * 128 + row;
+    const int part = mt * 4 + q, parts = mtiles * 4;
+    if (!mbar_wait(acc_bar, 0)) failed = true;
+    tc_fence_after();
+    if (!failed) {
+      const uint32_t trow = tmem_base + ((uint32_t)(32 * q) << 16);
+      float z[16];
+#pragma unroll
+      for (int c = 0; c < 16; ++c) z[c] = b2_s[c];
+      uint32_t v[32];
+      for (int ch = 0; ch < H / 32; ++ch) {
+        tc_ld32(trow + ch * 32, v);
+        float4* hout = reinterpret_cast<float4*>(sc.Hact + grow * H + ch * 32);
+#pragma unroll
+        for (int i4 = 0; i4 < 8; ++i4) {
+          float hv[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int col = ch * 32 + i4 * 4 + e;
+            hv[e] = fmaxf(__uint_as_float(v[i4 * 4 + e]) + b1_s[col], 0.f);
+            const float4* wr = reinterpret_cast<const float4*>(W2_s + col * 16);
+#pragma unroll
+            for (int c4 = 0; c4 < 4; ++c4) {
+              if (4 * c4 < C) {
+                const float4 w = wr[c4];
+                z[4 * c4] = fmaf(hv[e], w.x, z[4 * c4]); z[4 * c4 + 1] = fmaf(hv[e], w.y, z[4 * c4 + 1]);
+                z[4 * c4 + 2] = fmaf(hv[e], w.z, z[4 * c4 + 2]); z[4 * c4 + 3] = fmaf(hv[e], w.w, z[4 * c4 + 3]);
+              }
+            }
+          }
+          hout[i4] = make_float4(hv[0], hv[1], hv[2], hv[3]);
+        }
+      }
+      // softmax cross-entropy of this row; exponentials without the maximal class keep log(1+s)
+      // and p_max - 1 = -s/(1+s) accurate for wide margins
+      const int lab = label_s[row];
+      float zmax = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 16; ++c) { if (c >= C) z[c] = -INFINITY; zmax = fmaxf(zmax, z[c]); }
+      int cmax = 0;
+#pragma unroll
+      for (int c = 15; c >= 0; --c) if (c < C && z[c] == zmax) cmax = c;
+      float zl = 0.f;
+#pragma unroll
+      for (int c = 0; c < 16; ++c) if (c == lab) zl = z[c];
+      float sexcl = 0.f;
+#pragma unroll
+      for (int c = 0; c < 16; ++c) { z[c] = (c < C && c != cmax) ? expf(z[c] - zmax) : 0.f; sexcl += z[c]; }
+      const float ssum = 1.f + sexcl;
+      float d2[16];
+#pragma unroll
+      for (int c = 0; c < 16; ++c) {
+        float dl = 0.f;
+        if (c < C) {
+          if (c == cmax) dl = c == lab ? -sexcl / ssum : 1.f / ssum;
+          else dl = z[c] / ssum - (c == lab ? 1.f : 0.f);
+        }
+        d2[c] = dl;
+      }
+#pragma unroll
+      for (int c4 = 0; c4 < 4; ++c4)
+        reinterpret_cast<float4*>(sc.D2 + grow * 16)[c4] = make_float4(d2[4 * c4], d2[4 * c4 + 1], d2[4 * c4 + 2], d2[4 * c4 + 3]);
+      float rowloss = warp_sum(log1pf(sexcl) + (zmax - zl));
+      if (lane == 0) sc.loss_part[task * parts + part] = rowloss;
+
+      // second pass: delta1, its bf16 copy and its column sums over this warp's 32 rows
+      for (int ch = 0; ch < H / 32; ++ch) {
+        tc_ld32(trow + ch * 32, v);
+        float dv[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const int col = ch * 32 + i;
+          const float a1 = __uint_as_float(v[i]) + b1_s[col];
+          const float4* wr = reinterpret_cast<const float4*>(W2_s + col * 16);
+          float acc = 0.f;
+#pragma unroll
+          for (int c4 = 0; c4 < 4; ++c4) {
+            if (4 * c4 < C) {
+              const float4 w = wr[c4];
+              acc = fmaf(d2[4 * c4], w.x, acc); acc = fmaf(d2[4 * c4 + 1], w.y, acc);
+              acc = fmaf(d2[4 * c4 + 2], w.z, acc); acc = fmaf(d2[4 * c4 + 3], w.w, acc);
+            }
+          }
+          dv[i] = a1 > 0.f ? acc : 0.f;
+        }
+        uint4* dout = reinterpret_cast<uint4*>(sc.D1q + grow * H + ch * 32);
+#pragma unroll
+        for (int i8 = 0; i8 < 4; ++i8) {
+          uint32_t pk[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const __nv_bfloat162 b = __floats2bfloat162_rn(dv[i8 * 8 + 2 * e], dv[i8 * 8 + 2 * e + 1]);
+            pk[e] = *reinterpret_cast<const uint32_t*>(&b);
+          }
+          dout[i8] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
+        warp_transpose_reduce(dv, lane);
+        sc.db1_part[(task * parts + part) * H + ch * 32 + lane] = dv[0];
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tc_dealloc(tmem_base, tmem_cols);
+  if (failed && lane == 0) atomicExch(a.err, ERR_WAIT_TIMEOUT);
+}
+
+// ---- host: tensor maps ----------------------------------------------------------------------------
+typedef CUresult (*PFN_encodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                    const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline PFN_encodeTiled tc_encode_fn() {
+  static PFN_encodeTiled fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess && qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<PFN_encodeTiled>(p);
+  }
+  return fn;
+}
+
+// 2-D bf16 tensor [rows][cols] (cols contiguous), box = box_cols x box_rows, 128-byte swizzle
+inline bool tc_make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_cols, uint32_t box_rows) {
+  PFN_encodeTiled fn = tc_encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {cols * 2};
+  const cuuint32_t box[2] = {box_cols, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct MlpMaps { CUtensorMap tmX, tmW; bool ready = false; };
+
+inline cudaError_t run_mlp(NumericArgs& a, MlpScratch& s, MlpMaps& maps, int P, cudaStream_t stream, const char** why) {
+  *why = nullptr;
+  cudaError_t e;
+  const int n_halves = s.H > 256 ? 2 : 1;
+  if (!maps.ready) {
+    if (!tc_make_map(&maps.tmX, s.Xq, (uint64_t)s.n, (uint64_t)s.d, TC_BK, 1) ||
+        !tc_make_map(&maps.tmW, s.W1qT, (uint64_t)s.R * s.n_slots * s.H, (uint64_t)s.d, TC_BK, (uint32_t)(s.H / n_halves))) {
+      *why = "mlp: could not encode the TMA tensor maps";
+      return cudaSuccess;
+    }
+    maps.ready = true;
+  }
+  const TcLayout L = tc_forward_layout(s.H);
+  if ((e = cudaFuncSetAttribute(mlp_forward_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(mlp_dw1_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MLP_SMEM + 1024)) != cudaSuccess) return e;
+  MlpArgs g{};
+  g.na = a; g.sc = s; g.H = s.H; g.P = P;
+  const int mtiles = s.m / 128;
+  for (long long u = 0; u < a.iters; ++u) {
+    g.j = a.j0 + u;
+    mlp_forward_tc_kernel<<<a.R * s.Kmax * mtiles, TC_THREADS, L.total, stream>>>(maps.tmX, maps.tmW, g);
+    mlp_head_kernel<<<a.R * s.Kmax, 512, (size_t)s.m * 16 * 4, stream>>>(g);
+    mlp_dw1_update_kernel<<<a.R * (s.d / MLP_BM), 256, MLP_SMEM + 1024, stream>>>(g);
+    mlp_small_update_kernel<<<a.R, 256, 0, stream>>>(g);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+}  // namespace ssim

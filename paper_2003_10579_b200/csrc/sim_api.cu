@@ -11,7 +11,7 @@
 
 #include "linear_kernel.cuh"
 #include "softmax_kernel.cuh"
-#include "mlp_kernel.cuh"
+#include "mlp_tc_kernel.cuh"
 
 using namespace ssim;
 
@@ -62,6 +62,7 @@ struct sim_handle {
   float* w_state = nullptr;   // synchronous: [R][n_params]
   float* pool = nullptr;      // asynchronous: [R][n_slots][n_params]
   MlpScratch mlp{};
+  MlpMaps mlp_maps{};
   int* err = nullptr;
   TraceBuffers tr;
   bool poisoned = false;
@@ -390,7 +391,7 @@ sim_status sim_run(sim_handle* h, int64_t iters) {
                                  h->K_stride, h->R, h->n_slots, h->stream);
           if (ce == cudaSuccess) ce = mlp_after_set_params(h->mlp, h->pool, h->n_params, h->stream);
         }
-        if (ce == cudaSuccess) ce = run_mlp(a, h->mlp, h->P, h->stream, &why);
+        if (ce == cudaSuccess) ce = run_mlp(a, h->mlp, h->mlp_maps, h->P, h->stream, &why);
         if (ce == cudaSuccess && !h->is_async)   // synchronous variants ping-pong between two slots
           ce = cudaMemsetAsync(h->cur_slot, (int)((h->n_updates + iters) & 1), (size_t)h->R, h->stream);
         st = why ? fail(h, SIM_ERR_ARG, why) : SIM_OK;

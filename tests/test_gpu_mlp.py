@@ -60,7 +60,7 @@ def run_mlp_case(B, data, w0, *, variant, P, K, m, eta, R, J, kind="exp", mu=1.0
 
 
 @pytest.mark.parametrize("variant", list(core.VARIANTS))
-@pytest.mark.parametrize("d,H,C,m,K,P", [(128, 64, 4, 64, 2, 4), (256, 192, 10, 128, 3, 5), (3072, 512, 10, 128, 4, 16)])
+@pytest.mark.parametrize("d,H,C,m,K,P", [(128, 64, 4, 128, 2, 4), (256, 192, 10, 256, 3, 5), (3072, 512, 10, 128, 4, 16)])
 def test_mlp_variants_and_shapes(B, variant, d, H, C, m, K, P):
     data = inputs.make_mixture(4096, d, C, 0.5 if d < 1000 else 0.1, 95, "mlp2", H)
     w0 = inputs.mlp_init(d, H, C, 96)
@@ -70,9 +70,9 @@ def test_mlp_variants_and_shapes(B, variant, d, H, C, m, K, P):
 def test_mlp_growing_K_and_resume(B):
     data = inputs.make_mixture(2048, 128, 4, 0.5, 97, "mlp2", 64)
     w0 = inputs.mlp_init(128, 64, 4, 98)
-    run_mlp_case(B, data, w0, variant="kbatchasync", P=8, K=1, m=64, eta=0.02, R=4, J=60, K0=1, ti=2.0, chunks=(1, 7, 20))
+    run_mlp_case(B, data, w0, variant="kbatchasync", P=8, K=1, m=128, eta=0.02, R=4, J=60, K0=1, ti=2.0, chunks=(1, 7, 20))
     dev = to_device(data)
-    kw = dict(P=6, K=3, variant="kasync", delay_kind="exp", mu=1.0, eta=0.02, m=64, seed=1, n_replicas=3)
+    kw = dict(P=6, K=3, variant="kasync", delay_kind="exp", mu=1.0, eta=0.02, m=128, seed=1, n_replicas=3)
     a, b = B.Simulation(dev, **kw), B.Simulation(dev, **kw)
     for s in (a, b):
         s.set_params(torch.from_numpy(w0).cuda())
@@ -89,5 +89,5 @@ def test_mlp_growing_K_and_resume(B):
 def test_mlp_unsupported_shapes_are_refused(B):
     data = inputs.make_mixture(64, 128, 4, 0.5, 99, "mlp2", 100)
     with pytest.raises(B.SimError) as e:
-        B.Simulation(to_device(data), P=2, K=1, variant="ksync", delay_kind="exp", mu=1.0, eta=0.1, m=64, seed=0, n_replicas=1)
+        B.Simulation(to_device(data), P=2, K=1, variant="ksync", delay_kind="exp", mu=1.0, eta=0.1, m=128, seed=0, n_replicas=1)
     assert e.value.status == 1
