@@ -2,9 +2,12 @@
 // memory.
 //
 // One CTA per (replica, contributor, 128-sample block):  A1[128 x H] = bf16(X_b)[128 x d] bf16(W1)[d x H]
-//   warp 0   producer: TMA tensor loads into a ring of shared-memory stages (128-byte swizzle);
-//            the 128 gathered sample rows go in as 128 one-row boxes of 64 features, the W1 tile
-//            comes from the transposed bf16 shadow W1^T [H][d] (K-major B operand) as one or two boxes
+//   warp 0   B producer: TMA tensor loads of the W1 tile from the transposed bf16 shadow W1^T [H][d]
+//            (K-major B operand, 128-byte swizzle, one or two boxes per stage)
+//   warps 2-5  A producer during the main loop: the 128 gathered sample rows of a stage are 1024
+//            16-byte pieces, copied with cp.async into the same 128-byte-swizzle pattern (one-row
+//            TMA boxes of 128 B were limited by the TMA instruction rate), made visible to the
+//            tensor core's asynchronous proxy with a proxy fence before the stage is signalled
 //   warp 1   allocates tensor memory; one elected lane issues tcgen05.mma (M=128, N<=256, K=16)
 //            and commits stage-free / accumulator-ready mbarriers
 //   warps 2-5  epilogue: tcgen05.ld gives each thread one sample's full row of A1, so bias, relu,
@@ -132,7 +135,8 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
   const uint32_t acc_bar = bars + 8u * (2 * S);
 
   if (tid == 0) {
-    for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    // a stage is full after the TMA bytes of B (one arrival with expect_tx) and the 128 A-producer threads
+    for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1 + 128); mbar_init(empty_bar(s), 1); }
     mbar_init(acc_bar, 1);
     mbar_fence_init();
   }
@@ -162,24 +166,19 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
   bool failed = false;
 
   if (warp == 0) {
-    // ---- producer ----
+    // ---- B producer ----
     const int w_row0 = (int)(((size_t)r * sc.n_slots + snap) * H);
-    for (int kc = 0; kc < nk; ++kc) {
-      const int s = kc % S;
-      if (!mbar_wait(empty_bar(s), (uint32_t)(((kc / S) & 1) ^ 1))) { failed = true; break; }
-      const uint32_t As = base_addr + (uint32_t)s * L.stage_bytes, Bs = As + TC_A_BYTES;
-      if (lane == 0) {
-        mbar_arrive_expect_tx(full_bar(s), (uint32_t)L.stage_bytes);
+    if (lane == 0) {
+      for (int kc = 0; kc < nk; ++kc) {
+        const int s = kc % S;
+        if (!mbar_wait(empty_bar(s), (uint32_t)(((kc / S) & 1) ^ 1))) { failed = true; break; }
+        const uint32_t Bs = base_addr + (uint32_t)s * L.stage_bytes + TC_A_BYTES;
+        mbar_arrive_expect_tx(full_bar(s), (uint32_t)(H * 128));
         for (int hf = 0; hf < n_halves; ++hf)
           tma_load_2d(Bs + (uint32_t)hf * n_inst * 128, &tmW, kc * TC_BK, w_row0 + hf * n_inst, full_bar(s));
       }
-      __syncwarp();
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int row = lane + 32 * i;
-        tma_load_2d(As + (uint32_t)row * 128, &tmX, kc * TC_BK, rows_s[row], full_bar(s));
-      }
     }
+    __syncwarp();
   } else if (warp == 1) {
     // ---- MMA issuer ----
     const uint32_t idesc = tc_idesc(n_inst, 0, 0);
@@ -208,7 +207,33 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
     const int row = 32 * q + lane;
     const size_t grow = task * m + (size_t)mt * 128 + row;
     const int part = mt * 4 + q, parts = mtiles * 4;
-    if (!mbar_wait(acc_bar, 0)) failed = true;
+    // ---- A producer: thread t copies 16-byte piece (t & 7) of rows (t >> 3) + 16 i, i < 8 ----
+    {
+      const int t = tid - 64, ch = t & 7, row0 = t >> 3;
+      auto signal = [&](int kc2) {          // pieces of stage kc2 have landed: publish to the async proxy
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_arrive(full_bar(kc2 % S));
+      };
+      int signalled = 0;
+      for (int kc = 0; kc < nk && !failed; ++kc) {
+        const int s = kc % S;
+        if (!mbar_wait(empty_bar(s), (uint32_t)(((kc / S) & 1) ^ 1))) { failed = true; break; }
+        const uint32_t As = base_addr + (uint32_t)s * L.stage_bytes;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int rw = row0 + 16 * i;
+          cp_async16(As + rw * 128 + ((ch ^ (rw & 7)) << 4), sc.Xq + (size_t)rows_s[rw] * d + (size_t)kc * TC_BK + ch * 8);
+        }
+        cp_async_commit();
+        if (kc >= S - 1) {                  // the group issued S-1 iterations ago is complete
+          if (S == 2) cp_async_wait<1>(); else cp_async_wait<3>();
+          signal(signalled++);
+        }
+      }
+      cp_async_wait<0>();
+      if (!failed) while (signalled < nk) signal(signalled++);
+    }
+    if (!failed && !mbar_wait(acc_bar, 0)) failed = true;
     tc_fence_after();
     if (!failed) {
       const uint32_t trow = tmem_base + ((uint32_t)(32 * q) << 16);
