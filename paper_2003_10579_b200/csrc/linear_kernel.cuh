@@ -34,6 +34,7 @@ struct NumericArgs {
   int is_async;
   int n_slots;
   long long n_params;
+  long long slot_stride;     // floats between versions in the pool: n_params rounded up to a multiple of 4
   const uint16_t* K_used;    // schedule, see schedule_kernel.cuh
   const uint16_t* worker;
   const uint32_t* seq;

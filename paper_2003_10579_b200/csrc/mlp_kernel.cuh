@@ -13,10 +13,10 @@
 //             tcgen05 with the accumulator in tensor memory, then h = relu(A1 + b1), logits, softmax,
 //             delta2, delta1 = (delta2 W2^T) . [h > 0]; writes h, delta2, bf16(delta1), partial db1, loss
 //   head      one CTA per (replica, contributor): dW2 = h^T delta2, db2
-//   dw1       one CTA per (replica, 64-row slab of W1): accumulates X^T delta1 over all K m samples
-//             of the update (mma.sync m16n8k16, cp.async 3-stage ring, XOR-swizzled shared memory,
-//             ldmatrix) and applies W1 <- W1 - (eta/(K m)) dW1 in its epilogue (Eq. 2 / Eq. 3), writing
-//             the new version and its transposed bf16 shadow: dW1 never exists in memory
+//   dw1       (mlp_tc_kernel.cuh) one CTA per (replica, 128-row slab of W1): accumulates X^T delta1 over
+//             all K m samples of the update in tensor memory (tcgen05, MN-major operands) and applies
+//             W1 <- W1 - (eta/(K m)) dW1 in its epilogue (Eq. 2 / Eq. 3), writing the new version and
+//             its transposed bf16 shadow: dW1 never exists in memory
 //   small     b1, W2, b2 update from the partials (fixed summation order), loss record
 #pragma once
 #include <cuda_bf16.h>
@@ -46,17 +46,9 @@ struct MlpArgs {
   long long j;            // update being processed
 };
 
-constexpr int MLP_BM = 64;          // rows of the output tile per CTA
-constexpr int MLP_BK = 64;          // reduction chunk
-constexpr int MLP_PITCH_B = 1024;   // bytes per k-row of the B tile (H <= 512 bf16)
-constexpr int MLP_STAGE_A = MLP_BM * 128;              // 64 rows x 128 B
-constexpr int MLP_STAGE_B = MLP_BK * MLP_PITCH_B;      // 64 k-rows x 1024 B
-constexpr int MLP_STAGES = 3;
-constexpr int MLP_SMEM = MLP_STAGES * (MLP_STAGE_A + MLP_STAGE_B) + 1024;
-
 inline const char* mlp_shape_unsupported(int d, int H, int C, int m) {
   if (H < 64 || H > 512 || H % 64 != 0) return "mlp: hidden width must be a multiple of 64 in [64, 512]";
-  if (d % 64 != 0) return "mlp: d must be a multiple of 64";
+  if (d % 128 != 0) return "mlp: d must be a multiple of 128";
   if (m % 128 != 0) return "mlp: m must be a multiple of 128";
   if (C < 2 || C > 16) return "mlp: n_classes must be in [2, 16]";
   return nullptr;
@@ -69,20 +61,6 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
-__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
-}
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
-}
-__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
 
 // slot bookkeeping shared by the kernels: synchronous variants ping-pong between two slots
 __device__ __forceinline__ int mlp_cur_slot(const NumericArgs& a, int r, long long j) {
@@ -98,53 +76,18 @@ __device__ __forceinline__ int mlp_snap_slot(const NumericArgs& a, int r, long l
   return (int)a.snap_slot[((size_t)r * a.cap + j) * a.K_stride + l];
 }
 
-// One BK-deep step of the 64 x (8 warps x 64) tile: A fragments of the 4 row blocks, B fragments
-// of the warp's 8 column blocks, 32 MMAs.  A_KM: the A tile is stored [k][m] (transposed).
-template <bool A_KM>
-__device__ __forceinline__ void mlp_tile_mma(float (&acc)[4][8][4], uint32_t As, uint32_t Bs, int warp, int lane, int ncols) {
-  if (warp * 64 >= ncols) return;
-#pragma unroll
-  for (int k16 = 0; k16 < MLP_BK / 16; ++k16) {
-    uint32_t af[4][4];
-#pragma unroll
-    for (int mt = 0; mt < 4; ++mt) {
-      if (!A_KM) {
-        const int row = mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-        const int chunk = k16 * 2 + (lane >> 4);
-        ldmatrix_x4(af[mt], As + row * 128 + ((chunk ^ (row & 7)) << 4));
-      } else {
-        const int krow = k16 * 16 + (lane & 7) + (lane >> 4) * 8;
-        const int chunk = mt * 2 + ((lane >> 3) & 1);
-        ldmatrix_x4_trans(af[mt], As + krow * 128 + ((chunk ^ (krow & 7)) << 4));
-      }
-    }
-#pragma unroll
-    for (int np = 0; np < 4; ++np) {
-      uint32_t bf[4];
-      const int krow = k16 * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-      const int chunk = warp * 8 + np * 2 + (lane >> 4);
-      ldmatrix_x4_trans(bf, Bs + krow * MLP_PITCH_B + ((chunk ^ (krow & 7)) << 4));
-#pragma unroll
-      for (int mt = 0; mt < 4; ++mt) {
-        mma_bf16(acc[mt][2 * np], af[mt], bf[0], bf[1]);
-        mma_bf16(acc[mt][2 * np + 1], af[mt], bf[2], bf[3]);
-      }
-    }
-  }
-}
-
 // ---- data preparation ---------------------------------------------------------------------------
 __global__ void to_bf16_kernel(const float* src, __nv_bfloat16* dst, long long count) {
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < count; i += (long long)gridDim.x * blockDim.x)
     dst[i] = __float2bfloat16_rn(src[i]);
 }
 // transposed bf16 shadow (W1^T [H][d]) of W1 in pool slot `slot` of every replica
-__global__ void shadow_w1_kernel(const float* pool, __nv_bfloat16* W1qT, long long n_params, int d, int H, int n_slots, int slot, int R) {
+__global__ void shadow_w1_kernel(const float* pool, __nv_bfloat16* W1qT, long long slot_stride, int d, int H, int n_slots, int slot, int R) {
   const long long dH = (long long)d * H, total = dH * R;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
     const long long r = i / dH, p = i % dH;
     const long long n = p / d, k = p % d;       // output element (n, k) = W1[k][n]
-    W1qT[((size_t)r * n_slots + slot) * dH + p] = __float2bfloat16_rn(pool[((size_t)r * n_slots + slot) * n_params + k * H + n]);
+    W1qT[((size_t)r * n_slots + slot) * dH + p] = __float2bfloat16_rn(pool[((size_t)r * n_slots + slot) * slot_stride + k * H + n]);
   }
 }
 
@@ -183,109 +126,6 @@ __global__ void __launch_bounds__(512) mlp_head_kernel(MlpArgs g) {
   }
 }
 
-// ---- dW1 = X^T delta1 over all contributors of the update, fused with the W1 update ------------
-__global__ void __launch_bounds__(256, 1) mlp_dw1_update_kernel(MlpArgs g) {
-  const NumericArgs& a = g.na;
-  const MlpScratch& sc = g.sc;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int H = sc.H, d = sc.d, m = sc.m;
-  const int slabs = d / MLP_BM;
-  const int slab = blockIdx.x % slabs, r = blockIdx.x / slabs;
-  const long long j = g.j;
-  const int K = (int)a.K_used[(size_t)r * a.cap + j];
-  const uint32_t rid = a.replica_base + (uint32_t)r;
-  const long long dH = (long long)d * H;
-  const int blocks_per_task = m / MLP_BK;
-  const int nk = K * blocks_per_task;
-
-  extern __shared__ __align__(128) unsigned char smem[];
-  unsigned long long* rowptr_s = reinterpret_cast<unsigned long long*>(smem);   // [3 stages][64]... one set per stage
-  unsigned char* stages = smem + 2048;
-  const uint32_t stages_addr = smem_addr(stages);
-
-  auto draw_rows = [&](int kc) {   // sample rows of reduction block kc -> rowptr_s[kc % 3]
-    if (tid < MLP_BK) {
-      const int l = kc / blocks_per_task, blk = kc % blocks_per_task;
-      const size_t ent = ((size_t)r * a.cap + j) * a.K_stride + l;
-      uint32_t idx = draw_index(a.seed, rid, a.worker[ent], a.seq[ent], (uint32_t)(blk * MLP_BK + tid), a.n);
-      if ((uint64_t)idx >= a.n) { atomicExch(a.err, ERR_BAD_INDEX); idx = 0; }
-      rowptr_s[(kc % MLP_STAGES) * 64 + tid] = (unsigned long long)idx * (unsigned long long)d;
-    }
-  };
-  auto load_stage = [&](int kc) {
-    const int st = kc % MLP_STAGES;
-    const int l = kc / blocks_per_task, blk = kc % blocks_per_task;
-    const uint32_t As = stages_addr + st * (MLP_STAGE_A + MLP_STAGE_B);
-    const uint32_t Bs = As + MLP_STAGE_A;
-    // A tile stored [k = sample][m = 64 columns of this slab]
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      const int c = tid + 256 * i, krow = c >> 3, ch = c & 7;
-      cp_async16(As + krow * 128 + ((ch ^ (krow & 7)) << 4), sc.Xq + rowptr_s[st * 64 + krow] + (size_t)slab * MLP_BM + ch * 8);
-    }
-    const __nv_bfloat16* D1 = sc.D1q + (((size_t)r * sc.Kmax + l) * m + (size_t)blk * MLP_BK) * H;
-    const int nch = H / 8;
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const int c = tid + 256 * i, krow = c >> 6, ch = c & 63;
-      if (ch < nch) cp_async16(Bs + krow * MLP_PITCH_B + ((ch ^ (krow & 7)) << 4), D1 + (size_t)krow * H + ch * 8);
-    }
-  };
-
-  float acc[4][8][4];
-#pragma unroll
-  for (int mt = 0; mt < 4; ++mt)
-#pragma unroll
-    for (int nt = 0; nt < 8; ++nt)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) acc[mt][nt][e] = 0.f;
-
-  // the row indices of a block are drawn one iteration before its loads are issued
-  for (int s = 0; s < MLP_STAGES - 1; ++s) if (s < nk) draw_rows(s);
-  __syncthreads();
-  for (int s = 0; s < MLP_STAGES - 1; ++s) { if (s < nk) load_stage(s); cp_async_commit(); }
-  if (MLP_STAGES - 1 < nk) draw_rows(MLP_STAGES - 1);
-  for (int kc = 0; kc < nk; ++kc) {
-    cp_async_wait<MLP_STAGES - 2>();
-    __syncthreads();
-    if (kc + MLP_STAGES - 1 < nk) load_stage(kc + MLP_STAGES - 1);
-    cp_async_commit();
-    const int st = kc % MLP_STAGES;
-    const uint32_t As = stages_addr + st * (MLP_STAGE_A + MLP_STAGE_B);
-    mlp_tile_mma<true>(acc, As, As + MLP_STAGE_A, warp, lane, H);
-    // rows for block kc + STAGES go to slot kc % STAGES of rowptr_s: its last readers were the loads of
-    // block kc (issued two iterations ago); the next reader, load_stage(kc + STAGES), runs after the
-    // barrier at the top of the next iteration
-    if (kc + MLP_STAGES < nk) draw_rows(kc + MLP_STAGES);
-  }
-  cp_async_wait<0>();
-
-  // ---- epilogue: W1 <- W1 - (eta/(K m)) dW1 for this slab, new version + bf16 shadow ----
-  if (warp * 64 >= H) return;
-  const int cur = mlp_cur_slot(a, r, j), fresh = mlp_fresh_slot(a, r, j);
-  const float scale = (float)((double)a.eta / ((double)K * (double)m));
-  const float* wc = a.pool + ((size_t)r * a.n_slots + cur) * a.n_params;
-  float* wn = a.pool + ((size_t)r * a.n_slots + fresh) * a.n_params;
-  __nv_bfloat16* wq = sc.W1qT + ((size_t)r * sc.n_slots + fresh) * dH;   // [H][d]
-  const int g8 = lane >> 2, tig = lane & 3;
-#pragma unroll
-  for (int mt = 0; mt < 4; ++mt) {
-#pragma unroll
-    for (int rh = 0; rh < 2; ++rh) {
-      const size_t row = (size_t)slab * MLP_BM + mt * 16 + g8 + rh * 8;
-#pragma unroll
-      for (int nt = 0; nt < 8; ++nt) {
-        const int col = warp * 64 + nt * 8 + 2 * tig;
-        const float2 w = *reinterpret_cast<const float2*>(wc + row * H + col);
-        const float n0 = fmaf(-scale, acc[mt][nt][2 * rh], w.x), n1 = fmaf(-scale, acc[mt][nt][2 * rh + 1], w.y);
-        *reinterpret_cast<float2*>(wn + row * H + col) = make_float2(n0, n1);
-        wq[(size_t)col * d + row] = __float2bfloat16_rn(n0);
-        wq[(size_t)(col + 1) * d + row] = __float2bfloat16_rn(n1);
-      }
-    }
-  }
-}
-
 // ---- b1, W2, b2 update and the loss record -------------------------------------------------------
 __global__ void __launch_bounds__(256) mlp_small_update_kernel(MlpArgs g) {
   const NumericArgs& a = g.na;
@@ -297,8 +137,8 @@ __global__ void __launch_bounds__(256) mlp_small_update_kernel(MlpArgs g) {
   const long long dH = (long long)sc.d * H;
   const int cur = mlp_cur_slot(a, r, j), fresh = mlp_fresh_slot(a, r, j);
   const float scale = (float)((double)a.eta / ((double)K * (double)m));
-  const float* wc = a.pool + ((size_t)r * a.n_slots + cur) * a.n_params + dH;
-  float* wn = a.pool + ((size_t)r * a.n_slots + fresh) * a.n_params + dH;
+  const float* wc = a.pool + ((size_t)r * a.n_slots + cur) * a.slot_stride + dH;
+  float* wn = a.pool + ((size_t)r * a.n_slots + fresh) * a.slot_stride + dH;
   const int tail = H + H * C + C;
   for (int p = tid; p < tail; p += blockDim.x) {
     float gsum = 0.f;
@@ -349,8 +189,8 @@ inline cudaError_t mlp_scratch_alloc(MlpScratch& s, const float* X, long long n,
 }
 
 // after the initial parameters went into slot 0 of every replica
-inline cudaError_t mlp_after_set_params(MlpScratch& s, const float* pool, long long n_params, cudaStream_t stream) {
-  shadow_w1_kernel<<<1184, 256, 0, stream>>>(pool, s.W1qT, n_params, s.d, s.H, s.n_slots, 0, s.R);
+inline cudaError_t mlp_after_set_params(MlpScratch& s, const float* pool, long long slot_stride, cudaStream_t stream) {
+  shadow_w1_kernel<<<1184, 256, 0, stream>>>(pool, s.W1qT, slot_stride, s.d, s.H, s.n_slots, 0, s.R);
   return cudaGetLastError();
 }
 

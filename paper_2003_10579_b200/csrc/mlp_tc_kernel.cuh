@@ -111,7 +111,7 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
   const uint32_t rid = a.replica_base + (uint32_t)r;
   const size_t task = (size_t)r * sc.Kmax + l;
   const long long dH = (long long)d * H;
-  const float* wsnap = a.pool + ((size_t)r * a.n_slots + snap) * a.n_params;
+  const float* wsnap = a.pool + ((size_t)r * a.n_slots + snap) * a.slot_stride;
   const int n_halves = H > 256 ? 2 : 1;
   const int n_inst = H / n_halves;
   uint32_t tmem_cols = 32;
@@ -339,6 +339,191 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
   if (failed && lane == 0) atomicExch(a.err, ERR_WAIT_TIMEOUT);
 }
 
+
+// Shared-memory matrix descriptor, 128-byte swizzle, MN-major operand (the M or N index is the
+// contiguous one): 64-element (128-byte) runs along MN, 8 such k-rows form a 1024-byte atom;
+// the next 8 k-rows are `sbo` bytes on (stride byte offset), the next 64 MN elements `lbo` bytes on
+// (leading byte offset).
+__device__ __forceinline__ uint64_t tc_desc_mnmajor(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) | ((uint64_t)1 << 46) |
+         ((uint64_t)2 << 61);
+}
+
+struct TcDw1Layout { int stages, stage_bytes, off_rows, off_bars, off_tmem, total; };
+inline __host__ __device__ TcDw1Layout tc_dw1_layout(int H, int max_samples) {
+  TcDw1Layout L;
+  L.stage_bytes = TC_A_BYTES + H * 128;       // A: 64 samples x 128 features; B: 64 samples x H
+  L.stages = H <= 256 ? 4 : 2;
+  L.off_rows = L.stages * L.stage_bytes;
+  L.off_bars = L.off_rows + max_samples * 4;
+  L.off_tmem = L.off_bars + 8 * (2 * L.stages + 1);
+  L.total = L.off_tmem + 16 + 1024;
+  return L;
+}
+
+// dW1 = bf16(X)^T bf16(delta1) over all K m samples of the update, fused with the update of W1.
+// One CTA per (replica, 128-row slab of W1); the 128 x H accumulator lives in tensor memory.
+// Both operands are MN-major: a stage holds 64 samples; A = their features [slab*128, +128) as
+// gathered from the bf16 data set (cp.async by warps 2-5, written in the swizzled atom layout),
+// B = the same samples' bf16 delta1 rows (TMA boxes of 64 x 64).  The epilogue applies
+// W1 <- W1 - (eta/(K m)) dW1 (Eq. 2 / Eq. 3) and writes the new fp32 version and its transposed
+// bf16 shadow; dW1 itself never exists in memory.
+__global__ void __launch_bounds__(TC_THREADS, 1)
+mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
+  const NumericArgs& a = g.na;
+  const MlpScratch& sc = g.sc;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int H = sc.H, d = sc.d, m = sc.m;
+  const int slabs = d / 128;
+  const int slab = blockIdx.x % slabs, r = blockIdx.x / slabs;
+  const long long j = g.j;
+  const int K = (int)a.K_used[(size_t)r * a.cap + j];
+  const uint32_t rid = a.replica_base + (uint32_t)r;
+  const long long dH = (long long)d * H;
+  const int blocks_per_task = m / TC_BK;
+  const int nk = K * blocks_per_task;
+  const int n_halves = H > 256 ? 2 : 1;
+  const int n_inst = H / n_halves;
+  uint32_t tmem_cols = 32;
+  while ((int)tmem_cols < H) tmem_cols <<= 1;
+
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw_addr = smem_addr(smem_raw);
+  const uint32_t base_addr = (raw_addr + 1023u) & ~1023u;
+  unsigned char* base = smem_raw + (base_addr - raw_addr);
+  const TcDw1Layout L = tc_dw1_layout(H, sc.Kmax * m);
+  const int S = L.stages;
+  int* rows_s = reinterpret_cast<int*>(base + L.off_rows);
+  const uint32_t bars = base_addr + L.off_bars;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base + L.off_tmem);
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (S + s); };
+  const uint32_t acc_bar = bars + 8u * (2 * S);
+
+  if (tid == 0) {
+    for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1 + 128); mbar_init(empty_bar(s), 1); }
+    mbar_init(acc_bar, 1);
+    mbar_fence_init();
+  }
+  if (warp == 1) tc_alloc(smem_addr(tmem_slot), tmem_cols);
+  for (int i = tid; i < K * m; i += TC_THREADS) {      // sample rows of the whole update, contributor-major
+    const int l = i / m, q = i % m;
+    const size_t ent = ((size_t)r * a.cap + j) * a.K_stride + l;
+    uint32_t idx = draw_index(a.seed, rid, a.worker[ent], a.seq[ent], (uint32_t)q, a.n);
+    if ((uint64_t)idx >= a.n) { atomicExch(a.err, ERR_BAD_INDEX); idx = 0; }
+    rows_s[i] = (int)idx;
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  bool failed = false;
+  const uint32_t ATOM = 8192;     // one 64-wide MN block of a 64-sample stage: 64 k-rows x 128 B
+
+  if (warp == 0) {
+    // ---- B producer: delta1 rows of 64 samples, H/64 boxes of 64 x 64 ----
+    if (lane == 0) {
+      for (int kc = 0; kc < nk; ++kc) {
+        const int s = kc % S;
+        if (!mbar_wait(empty_bar(s), (uint32_t)(((kc / S) & 1) ^ 1))) { failed = true; break; }
+        const uint32_t Bs = base_addr + (uint32_t)s * L.stage_bytes + TC_A_BYTES;
+        const int l = kc / blocks_per_task, blk = kc % blocks_per_task;
+        const int row0 = (int)(((size_t)r * sc.Kmax + l) * m + (size_t)blk * TC_BK);
+        mbar_arrive_expect_tx(full_bar(s), (uint32_t)(H * 128));
+        for (int b = 0; b < H / 64; ++b) tma_load_2d(Bs + (uint32_t)b * ATOM, &tmD, b * 64, row0, full_bar(s));
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ---- MMA issuer ----
+    const uint32_t idesc = tc_idesc(n_inst, 1, 1);
+    const uint32_t lbo = ATOM, sbo = 1024u;   // next 64 MN elements: one atom block on; next 8 samples: 1024 B on
+    for (int kc = 0; kc < nk; ++kc) {
+      const int s = kc % S;
+      if (!mbar_wait(full_bar(s), (uint32_t)((kc / S) & 1))) { failed = true; break; }
+      tc_fence_after();
+      if (lane == 0) {
+        const uint32_t As = base_addr + (uint32_t)s * L.stage_bytes, Bs = As + TC_A_BYTES;
+#pragma unroll
+        for (int k16 = 0; k16 < TC_BK / 16; ++k16) {      // 16 samples = two 8-row groups = 2048 B
+          const uint64_t ad = tc_desc_mnmajor(As + k16 * 2048, lbo, sbo);
+          for (int hf = 0; hf < n_halves; ++hf) {
+            const uint64_t bd = tc_desc_mnmajor(Bs + (uint32_t)hf * (n_inst / 64) * ATOM + k16 * 2048, lbo, sbo);
+            tc_mma_bf16(tmem_base + (uint32_t)hf * n_inst, ad, bd, idesc, (kc > 0 || k16 > 0) ? 1u : 0u);
+          }
+        }
+        tc_commit(empty_bar(s));
+        if (kc == nk - 1) tc_commit(acc_bar);
+      }
+      __syncwarp();
+    }
+  } else {
+    // ---- A producer: thread t copies 16-byte piece (t & 15) of sample rows (t >> 4) + 8 i, i < 8 ----
+    {
+      const int t = tid - 64, piece = t & 15, k0 = t >> 4;
+      auto signal = [&](int kc2) {
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_arrive(full_bar(kc2 % S));
+      };
+      int signalled = 0;
+      for (int kc = 0; kc < nk && !failed; ++kc) {
+        const int s = kc % S;
+        if (!mbar_wait(empty_bar(s), (uint32_t)(((kc / S) & 1) ^ 1))) { failed = true; break; }
+        const uint32_t As = base_addr + (uint32_t)s * L.stage_bytes + (uint32_t)(piece >> 3) * ATOM;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int k = k0 + 8 * i;
+          cp_async16(As + (k >> 3) * 1024 + (k & 7) * 128 + (((piece & 7) ^ (k & 7)) << 4),
+                     sc.Xq + (size_t)rows_s[kc * TC_BK + k] * d + (size_t)slab * 128 + piece * 8);
+        }
+        cp_async_commit();
+        if (kc >= S - 1) {
+          if (S == 2) cp_async_wait<1>(); else cp_async_wait<3>();
+          signal(signalled++);
+        }
+      }
+      cp_async_wait<0>();
+      if (!failed) while (signalled < nk) signal(signalled++);
+    }
+    // ---- epilogue: thread = one row of W1 ----
+    const int q = warp & 3;
+    const size_t row = (size_t)slab * 128 + 32 * q + lane;
+    if (!failed && !mbar_wait(acc_bar, 0)) failed = true;
+    tc_fence_after();
+    if (!failed) {
+      const uint32_t trow = tmem_base + ((uint32_t)(32 * q) << 16);
+      const int cur = mlp_cur_slot(a, r, j), fresh = mlp_fresh_slot(a, r, j);
+      const float scale = (float)((double)a.eta / ((double)K * (double)m));
+      const float* wc = a.pool + ((size_t)r * a.n_slots + cur) * a.slot_stride + row * H;
+      float* wn = a.pool + ((size_t)r * a.n_slots + fresh) * a.slot_stride + row * H;
+      __nv_bfloat16* wq = sc.W1qT + ((size_t)r * sc.n_slots + fresh) * dH + row;   // [H][d], this row's column
+      uint32_t v[32];
+      for (int ch = 0; ch < H / 32; ++ch) {
+        tc_ld32(trow + ch * 32, v);
+#pragma unroll
+        for (int i4 = 0; i4 < 8; ++i4) {
+          float4 w = reinterpret_cast<const float4*>(wc + ch * 32)[i4];
+          w.x = fmaf(-scale, __uint_as_float(v[4 * i4]), w.x);
+          w.y = fmaf(-scale, __uint_as_float(v[4 * i4 + 1]), w.y);
+          w.z = fmaf(-scale, __uint_as_float(v[4 * i4 + 2]), w.z);
+          w.w = fmaf(-scale, __uint_as_float(v[4 * i4 + 3]), w.w);
+          reinterpret_cast<float4*>(wn + ch * 32)[i4] = w;
+          const int col = ch * 32 + 4 * i4;
+          wq[(size_t)col * d] = __float2bfloat16_rn(w.x);
+          wq[(size_t)(col + 1) * d] = __float2bfloat16_rn(w.y);
+          wq[(size_t)(col + 2) * d] = __float2bfloat16_rn(w.z);
+          wq[(size_t)(col + 3) * d] = __float2bfloat16_rn(w.w);
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tc_dealloc(tmem_base, tmem_cols);
+  if (failed && lane == 0) atomicExch(a.err, ERR_WAIT_TIMEOUT);
+}
+
 // ---- host: tensor maps ----------------------------------------------------------------------------
 typedef CUresult (*PFN_encodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                     const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -367,7 +552,7 @@ inline bool tc_make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-struct MlpMaps { CUtensorMap tmX, tmW; bool ready = false; };
+struct MlpMaps { CUtensorMap tmX, tmW, tmD; bool ready = false; };
 
 inline cudaError_t run_mlp(NumericArgs& a, MlpScratch& s, MlpMaps& maps, int P, cudaStream_t stream, const char** why) {
   *why = nullptr;
@@ -375,7 +560,8 @@ inline cudaError_t run_mlp(NumericArgs& a, MlpScratch& s, MlpMaps& maps, int P, 
   const int n_halves = s.H > 256 ? 2 : 1;
   if (!maps.ready) {
     if (!tc_make_map(&maps.tmX, s.Xq, (uint64_t)s.n, (uint64_t)s.d, TC_BK, 1) ||
-        !tc_make_map(&maps.tmW, s.W1qT, (uint64_t)s.R * s.n_slots * s.H, (uint64_t)s.d, TC_BK, (uint32_t)(s.H / n_halves))) {
+        !tc_make_map(&maps.tmW, s.W1qT, (uint64_t)s.R * s.n_slots * s.H, (uint64_t)s.d, TC_BK, (uint32_t)(s.H / n_halves)) ||
+        !tc_make_map(&maps.tmD, s.D1q, (uint64_t)s.R * s.Kmax * s.m, (uint64_t)s.H, 64, 64)) {
       *why = "mlp: could not encode the TMA tensor maps";
       return cudaSuccess;
     }
@@ -383,7 +569,9 @@ inline cudaError_t run_mlp(NumericArgs& a, MlpScratch& s, MlpMaps& maps, int P, 
   }
   const TcLayout L = tc_forward_layout(s.H);
   if ((e = cudaFuncSetAttribute(mlp_forward_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total)) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(mlp_dw1_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MLP_SMEM + 1024)) != cudaSuccess) return e;
+  const TcDw1Layout LD = tc_dw1_layout(s.H, s.Kmax * s.m);
+  if (LD.total > (227 << 10)) { *why = "mlp: K_max * m too large for the dW1 kernel's row table"; return cudaSuccess; }
+  if ((e = cudaFuncSetAttribute(mlp_dw1_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, LD.total)) != cudaSuccess) return e;
   MlpArgs g{};
   g.na = a; g.sc = s; g.H = s.H; g.P = P;
   const int mtiles = s.m / 128;
@@ -391,7 +579,7 @@ inline cudaError_t run_mlp(NumericArgs& a, MlpScratch& s, MlpMaps& maps, int P, 
     g.j = a.j0 + u;
     mlp_forward_tc_kernel<<<a.R * s.Kmax * mtiles, TC_THREADS, L.total, stream>>>(maps.tmX, maps.tmW, g);
     mlp_head_kernel<<<a.R * s.Kmax, 512, (size_t)s.m * 16 * 4, stream>>>(g);
-    mlp_dw1_update_kernel<<<a.R * (s.d / MLP_BM), 256, MLP_SMEM + 1024, stream>>>(g);
+    mlp_dw1_tc_kernel<<<a.R * (s.d / 128), TC_THREADS, LD.total, stream>>>(maps.tmD, g);
     mlp_small_update_kernel<<<a.R, 256, 0, stream>>>(g);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }

@@ -49,6 +49,7 @@ struct sim_handle {
   bool uses_pool = false;     // parameters live in a version pool (asynchronous variants, and the MLP always)
   int n_slots = 0;
   long long n_params = 0;
+  long long slot_stride = 0;  // floats between versions in the pool (16-byte aligned slots)
   long long n_updates = 0, cap = 0;
   int tune_stages = 0, tune_rows = 0, tune_threads = 0;
   // device state
@@ -119,11 +120,11 @@ __global__ void broadcast_params_kernel(const float* w0, float* dst, long long n
   }
 }
 
-__global__ void gather_params_kernel(const float* pool, const uint8_t* cur_slot, float* out, long long n_params, int n_slots, int R) {
+__global__ void gather_params_kernel(const float* pool, const uint8_t* cur_slot, float* out, long long n_params, long long slot_stride, int n_slots, int R) {
   const long long total = n_params * R;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
     const long long r = i / n_params, p = i % n_params;
-    out[i] = pool[(r * n_slots + cur_slot[r]) * n_params + p];
+    out[i] = pool[(r * n_slots + cur_slot[r]) * slot_stride + p];
   }
 }
 
@@ -277,6 +278,7 @@ sim_status sim_create(const sim_problem* problem, int32_t P, int32_t K, sim_vari
   h->uses_pool = h->is_async || prob.model == SIM_MLP2;
   h->n_slots = h->is_async ? P + 2 : (prob.model == SIM_MLP2 ? 2 : 0);
   h->n_params = model_params(prob);
+  h->slot_stride = (h->n_params + 3) & ~3ll;
 
   cudaError_t e = cudaGetDevice(&h->device);
   const size_t RP = (size_t)h->R * P;
@@ -289,7 +291,7 @@ sim_status sim_create(const sim_problem* problem, int32_t P, int32_t K, sim_vari
   if (e == cudaSuccess) e = dev_alloc(&h->clock, (size_t)h->R, h->stream);
   if (e == cudaSuccess) e = dev_alloc(&h->err, 1, h->stream);
   if (e == cudaSuccess && h->n_params > 0) {
-    if (h->uses_pool) e = dev_alloc(&h->pool, (size_t)h->R * h->n_slots * h->n_params, h->stream);
+    if (h->uses_pool) e = dev_alloc(&h->pool, (size_t)h->R * h->n_slots * h->slot_stride, h->stream);
     else e = dev_alloc(&h->w_state, (size_t)h->R * h->n_params, h->stream);
   }
   if (e != cudaSuccess) {
@@ -310,7 +312,7 @@ sim_status sim_set_params(sim_handle* h, const float* w0) {
   if (h->n_updates > 0) return fail(h, SIM_ERR_STATE, "sim_set_params is only allowed before the first sim_run");
   if (h->n_params == 0) return SIM_OK;
   float* dst = h->uses_pool ? h->pool : h->w_state;
-  const long long stride = h->uses_pool ? (long long)h->n_slots * h->n_params : h->n_params;
+  const long long stride = h->uses_pool ? (long long)h->n_slots * h->slot_stride : h->n_params;
   broadcast_params_kernel<<<1184, 256, 0, h->stream>>>(w0, dst, h->n_params, stride, h->R);
   CUDA_TRY(h, cudaGetLastError());
   // the caller's buffer is read by enqueued work: finish it before returning
@@ -373,7 +375,7 @@ sim_status sim_run(sim_handle* h, int64_t iters) {
     a.w_ref = h->prob.w_ref; a.n = (uint64_t)h->prob.n; a.d = h->prob.d; a.m = h->m; a.model = (int)h->prob.model;
     a.n_classes = h->prob.n_classes; a.eta = h->eta; a.seed = h->seed; a.replica_base = h->replica_base; a.R = h->R;
     a.j0 = h->n_updates; a.iters = iters; a.cap = h->cap; a.K_stride = h->K_stride; a.is_async = h->is_async ? 1 : 0;
-    a.n_slots = h->n_slots; a.n_params = h->n_params;
+    a.n_slots = h->n_slots; a.n_params = h->n_params; a.slot_stride = h->slot_stride;
     a.K_used = h->tr.K_used; a.worker = h->tr.worker; a.seq = h->tr.seq; a.snap_slot = h->tr.snap_slot;
     a.new_slot = h->tr.new_slot; a.begin_slot = h->begin_slot; a.loss = h->tr.loss; a.dist2 = h->tr.dist2;
     a.w_state = h->w_state; a.pool = h->pool; a.err = h->err;
@@ -389,7 +391,7 @@ sim_status sim_run(sim_handle* h, int64_t iters) {
         if (!h->mlp.Xq) {   // first run: bf16 copy of the data, per-update scratch, bf16 shadow of the initial W1
           ce = mlp_scratch_alloc(h->mlp, h->prob.X, h->prob.n, h->prob.d, h->prob.hidden, h->prob.n_classes, h->m,
                                  h->K_stride, h->R, h->n_slots, h->stream);
-          if (ce == cudaSuccess) ce = mlp_after_set_params(h->mlp, h->pool, h->n_params, h->stream);
+          if (ce == cudaSuccess) ce = mlp_after_set_params(h->mlp, h->pool, h->slot_stride, h->stream);
         }
         if (ce == cudaSuccess) ce = run_mlp(a, h->mlp, h->mlp_maps, h->P, h->stream, &why);
         if (ce == cudaSuccess && !h->is_async)   // synchronous variants ping-pong between two slots
@@ -445,7 +447,7 @@ sim_status sim_get_params(const sim_handle* h, float* w) {
   if (st != SIM_OK) return st;
   if (h->n_params == 0) return SIM_OK;
   if (h->uses_pool) {
-    gather_params_kernel<<<1184, 256, 0, h->stream>>>(h->pool, h->cur_slot, w, h->n_params, h->n_slots, h->R);
+    gather_params_kernel<<<1184, 256, 0, h->stream>>>(h->pool, h->cur_slot, w, h->n_params, h->slot_stride, h->n_slots, h->R);
     CUDA_TRY(h, cudaGetLastError());
   } else {
     CUDA_TRY(h, cudaMemcpyAsync(w, h->w_state, (size_t)h->R * h->n_params * sizeof(float), cudaMemcpyDeviceToDevice, h->stream));
