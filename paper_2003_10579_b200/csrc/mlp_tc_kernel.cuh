@@ -32,6 +32,7 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_alloc(uint32_t smem_dst, uint32_t ncols) {
@@ -350,10 +351,15 @@ __device__ __forceinline__ uint64_t tc_desc_mnmajor(uint32_t saddr, uint32_t lbo
 }
 
 struct TcDw1Layout { int stages, stage_bytes, off_rows, off_bars, off_tmem, total; };
+// columns of W1 handled by one CTA of the dW1 kernel: 128 where H allows, so that three CTAs
+// (128 tensor-memory columns and ~70 KB of shared memory each) share an SM and one CTA's
+// row-per-thread epilogue overlaps the others' loads
+inline __host__ __device__ int tc_dw1_cols(int H) { return H % 128 == 0 ? 128 : 64; }
 inline __host__ __device__ TcDw1Layout tc_dw1_layout(int H, int max_samples) {
   TcDw1Layout L;
-  L.stage_bytes = TC_A_BYTES + H * 128;       // A: 64 samples x 128 features; B: 64 samples x H
-  L.stages = H <= 256 ? 4 : 2;
+  const int Hc = tc_dw1_cols(H);
+  L.stage_bytes = TC_A_BYTES + Hc * 128;      // A: 64 samples x 128 features; B: 64 samples x Hc
+  L.stages = 2;
   L.off_rows = L.stages * L.stage_bytes;
   L.off_bars = L.off_rows + max_samples * 4;
   L.off_tmem = L.off_bars + 8 * (2 * L.stages + 1);
@@ -362,30 +368,33 @@ inline __host__ __device__ TcDw1Layout tc_dw1_layout(int H, int max_samples) {
 }
 
 // dW1 = bf16(X)^T bf16(delta1) over all K m samples of the update, fused with the update of W1.
-// One CTA per (replica, 128-row slab of W1); the 128 x H accumulator lives in tensor memory.
+// One CTA per (replica, 128-row slab of W1, block of Hc columns); the 128 x Hc accumulator lives in
+// tensor memory.
 // Both operands are MN-major: a stage holds 64 samples; A = their features [slab*128, +128) as
 // gathered from the bf16 data set (cp.async by warps 2-5, written in the swizzled atom layout),
 // B = the same samples' bf16 delta1 rows (TMA boxes of 64 x 64).  The epilogue applies
 // W1 <- W1 - (eta/(K m)) dW1 (Eq. 2 / Eq. 3) and writes the new fp32 version and its transposed
 // bf16 shadow; dW1 itself never exists in memory.
-__global__ void __launch_bounds__(TC_THREADS, 1)
+__global__ void __launch_bounds__(TC_THREADS)
 mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
   const NumericArgs& a = g.na;
   const MlpScratch& sc = g.sc;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int H = sc.H, d = sc.d, m = sc.m;
   const int slabs = d / 128;
-  const int slab = blockIdx.x % slabs, r = blockIdx.x / slabs;
+  const int Hc = tc_dw1_cols(H), splits = H / Hc;
+  const int cs = blockIdx.x % splits;                 // column block
+  const int slab = (blockIdx.x / splits) % slabs, r = blockIdx.x / (splits * slabs);
+  const int col0 = cs * Hc;
   const long long j = g.j;
   const int K = (int)a.K_used[(size_t)r * a.cap + j];
   const uint32_t rid = a.replica_base + (uint32_t)r;
   const long long dH = (long long)d * H;
   const int blocks_per_task = m / TC_BK;
   const int nk = K * blocks_per_task;
-  const int n_halves = H > 256 ? 2 : 1;
-  const int n_inst = H / n_halves;
+  const int n_inst = Hc;                              // <= 128: one MMA covers the CTA's columns
   uint32_t tmem_cols = 32;
-  while ((int)tmem_cols < H) tmem_cols <<= 1;
+  while ((int)tmem_cols < Hc) tmem_cols <<= 1;
 
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw_addr = smem_addr(smem_raw);
@@ -429,8 +438,8 @@ mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
         const uint32_t Bs = base_addr + (uint32_t)s * L.stage_bytes + TC_A_BYTES;
         const int l = kc / blocks_per_task, blk = kc % blocks_per_task;
         const int row0 = (int)(((size_t)r * sc.Kmax + l) * m + (size_t)blk * TC_BK);
-        mbar_arrive_expect_tx(full_bar(s), (uint32_t)(H * 128));
-        for (int b = 0; b < H / 64; ++b) tma_load_2d(Bs + (uint32_t)b * ATOM, &tmD, b * 64, row0, full_bar(s));
+        mbar_arrive_expect_tx(full_bar(s), (uint32_t)(Hc * 128));
+        for (int b = 0; b < Hc / 64; ++b) tma_load_2d(Bs + (uint32_t)b * ATOM, &tmD, col0 + b * 64, row0, full_bar(s));
       }
     }
     __syncwarp();
@@ -447,10 +456,8 @@ mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
 #pragma unroll
         for (int k16 = 0; k16 < TC_BK / 16; ++k16) {      // 16 samples = two 8-row groups = 2048 B
           const uint64_t ad = tc_desc_mnmajor(As + k16 * 2048, lbo, sbo);
-          for (int hf = 0; hf < n_halves; ++hf) {
-            const uint64_t bd = tc_desc_mnmajor(Bs + (uint32_t)hf * (n_inst / 64) * ATOM + k16 * 2048, lbo, sbo);
-            tc_mma_bf16(tmem_base + (uint32_t)hf * n_inst, ad, bd, idesc, (kc > 0 || k16 > 0) ? 1u : 0u);
-          }
+          const uint64_t bd = tc_desc_mnmajor(Bs + k16 * 2048, lbo, sbo);
+          tc_mma_bf16(tmem_base, ad, bd, idesc, (kc > 0 || k16 > 0) ? 1u : 0u);
         }
         tc_commit(empty_bar(s));
         if (kc == nk - 1) tc_commit(acc_bar);
@@ -458,6 +465,17 @@ mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
       __syncwarp();
     }
   } else {
+    // The CTA's whole working set is known now: ask L2 for it at once (the 256-byte feature slices
+    // of all K m sample rows and this thread's row of w_j), so that the short software pipeline
+    // below runs against L2 latency instead of one DRAM round trip per stage.
+    {
+      const int t = tid - 64;
+      for (int i = t; i < 2 * K * m; i += 128)
+        prefetch_l2(sc.Xq + (size_t)rows_s[i >> 1] * d + (size_t)slab * 128 + (i & 1) * 64);
+      const float* wrow = a.pool + ((size_t)r * a.n_slots + mlp_cur_slot(a, r, j)) * a.slot_stride +
+                          ((size_t)slab * 128 + 32 * (warp & 3) + lane) * H + col0;
+      for (int i = 0; i < Hc / 32; ++i) prefetch_l2(wrow + i * 32);
+    }
     // ---- A producer: thread t copies 16-byte piece (t & 15) of sample rows (t >> 4) + 8 i, i < 8 ----
     {
       const int t = tid - 64, piece = t & 15, k0 = t >> 4;
@@ -494,11 +512,11 @@ mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
       const uint32_t trow = tmem_base + ((uint32_t)(32 * q) << 16);
       const int cur = mlp_cur_slot(a, r, j), fresh = mlp_fresh_slot(a, r, j);
       const float scale = (float)((double)a.eta / ((double)K * (double)m));
-      const float* wc = a.pool + ((size_t)r * a.n_slots + cur) * a.slot_stride + row * H;
-      float* wn = a.pool + ((size_t)r * a.n_slots + fresh) * a.slot_stride + row * H;
-      __nv_bfloat16* wq = sc.W1qT + ((size_t)r * sc.n_slots + fresh) * dH + row;   // [H][d], this row's column
+      const float* wc = a.pool + ((size_t)r * a.n_slots + cur) * a.slot_stride + row * H + col0;
+      float* wn = a.pool + ((size_t)r * a.n_slots + fresh) * a.slot_stride + row * H + col0;
+      __nv_bfloat16* wq = sc.W1qT + ((size_t)r * sc.n_slots + fresh) * dH + (size_t)col0 * d + row;   // [H][d], this row's column
       uint32_t v[32];
-      for (int ch = 0; ch < H / 32; ++ch) {
+      for (int ch = 0; ch < Hc / 32; ++ch) {
         tc_ld32(trow + ch * 32, v);
 #pragma unroll
         for (int i4 = 0; i4 < 8; ++i4) {
@@ -579,7 +597,7 @@ inline cudaError_t run_mlp(NumericArgs& a, MlpScratch& s, MlpMaps& maps, int P, 
     g.j = a.j0 + u;
     mlp_forward_tc_kernel<<<a.R * s.Kmax * mtiles, TC_THREADS, L.total, stream>>>(maps.tmX, maps.tmW, g);
     mlp_head_kernel<<<a.R * s.Kmax, 512, (size_t)s.m * 16 * 4, stream>>>(g);
-    mlp_dw1_tc_kernel<<<a.R * (s.d / 128), TC_THREADS, LD.total, stream>>>(maps.tmD, g);
+    mlp_dw1_tc_kernel<<<a.R * (s.d / 128) * (s.H / tc_dw1_cols(s.H)), TC_THREADS, LD.total, stream>>>(maps.tmD, g);
     mlp_small_update_kernel<<<a.R, 256, 0, stream>>>(g);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
