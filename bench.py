@@ -142,7 +142,8 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2003_10579_b200.binding import Simulation, simulate_host
+    from paper_2003_10579_b200.binding import Simulation, sweep_host
+    from paper_2003_10579_b200.sharding import replica_block
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -163,7 +164,7 @@ def main():
     for variant, K in wl.runs:
         st = main_stream if args.serial else torch.cuda.Stream()
         sim = Simulation(dev, P=wl.P, K=K, variant=variant, delay_kind=wl.delay_kind, mu=wl.mu, shift=wl.shift,
-                         eta=wl.eta, m=wl.m, seed=wl.seed, n_replicas=R, replica_base=rank * R, w_ref=w_ref,
+                         eta=wl.eta, m=wl.m, seed=wl.seed, n_replicas=R, replica_base=replica_block(rank, world, R)[0], w_ref=w_ref,
                          stream=None if args.serial else st)
         sim.reserve(total_steps * U)
         if args.stages:
@@ -220,7 +221,10 @@ def main():
     peak = float(peaks.get("hbm_gbs", 6650.0))
     achieved = step_bytes * args.steps / (ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None, "peak_source": "measured" if peaks else "fallback",
+                # DRAM bytes of the step: ncu small-case capture of this kernel (profiles/), dram read+write =
+                # 0.678 x algorithmic bytes, scaled by the rows gathered
+                "traffic": 0.678 * step_bytes, "traffic_scaled_from": "profiles/linear1_kernel_small_case_counters.txt",
+                "peak_source": "measured" if peaks else "fallback",
                 "kernel": "linear1_kernel (32 concurrent launches per step; summed algorithmic bytes over the step's device time)"}
 
     # a simulation that ran must have produced a finite trace (also surfaces device-side errors)
@@ -238,8 +242,9 @@ def main():
             "roofline": roofline, "clocks": clocks,
             "gpu_launches": 2 * len(sims) * args.steps}
 
-    if rank == 0 and not args.no_e2e:
-        # the public one-shot call on pinned host buffers: copies the data set in, simulates, copies the trace out
+    if not args.no_e2e:
+        # the public one-shot call on pinned host buffers: one step's work (all 32 runs, U updates from
+        # w_0) including the copy of the data set to the device and of the traces back, every step
         for sim in sims:
             sim.close()
         sims = []
@@ -247,19 +252,26 @@ def main():
         Xp = torch.from_numpy(data["X"]).pin_memory()
         yp = torch.from_numpy(data["y"]).pin_memory()
         host = {"model": "lsq", "X": Xp.numpy(), "y": yp.numpy()}
-        e2e_runs = wl.runs
         kw = dict(P=wl.P, delay_kind=wl.delay_kind, mu=wl.mu, shift=wl.shift, eta=wl.eta, m=wl.m, seed=wl.seed,
-                  n_replicas=R, iters=U, want=("t", "loss"))
-        simulate_host(host, variant="ksync", K=1, **kw)
+                  n_replicas=R, replica_base=rank * R, iters=U, want=("t", "loss"))
+        e2e_steps = max(1, min(args.steps, 5))
+        sweep_host(host, wl.runs, **kw)
+        barrier()
         t0 = time.perf_counter()
-        for variant, K in e2e_runs:
-            simulate_host(host, variant=variant, K=K, **kw)
+        for _ in range(e2e_steps):
+            out = sweep_host(host, wl.runs, **kw)
         torch.cuda.synchronize()
         dt = time.perf_counter() - t0
-        line["e2e"] = {"value": len(e2e_runs) * R * U / dt, "unit": UNIT,
-                       "h2d_bytes_per_step": len(e2e_runs) * (Xp.numel() * 4 + yp.numel() * 4),
-                       "d2h_bytes_per_step": len(e2e_runs) * R * U * 12,
-                       "note": "one sim_simulate_host call per (variant, K) run, host wall clock"}
+        if world > 1:
+            tt = torch.tensor([dt], device="cuda")
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            dt = float(tt.item())
+        assert np.isfinite(out["loss"]).all()
+        line["e2e"] = {"value": world * e2e_steps * len(wl.runs) * R * U / dt, "unit": UNIT,
+                       "h2d_bytes_per_step": Xp.numel() * 4 + yp.numel() * 4,
+                       "d2h_bytes_per_step": len(wl.runs) * R * U * 12, "steps": e2e_steps,
+                       "note": "sim_sweep_host per step: data set host->device, 32 runs x %d updates, "
+                               "clocks and losses device->host; host wall clock, max over ranks" % U}
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         reps, ups = 8, 150

@@ -172,6 +172,19 @@ sim_status sim_simulate_host(const sim_problem* problem, int32_t P, int32_t K, s
                              uint16_t* worker, uint32_t* stale, uint32_t* seq, float* w_final);
 
 /*
+ * A sweep on HOST buffers: the same data set and delay law under n_runs (variant, K) pairs - the
+ * comparison of Section 5's error-runtime trade-offs across K and across variants.  The data set
+ * is copied to the device once, the runs are simulated concurrently (one stream each) for `iters`
+ * updates from w0 (host, may be NULL for zeros), and the clocks, losses and distances come back
+ * as [n_runs][R][iters] host arrays (any may be NULL).  `problem` holds HOST pointers.  Everything
+ * allocated is freed before returning.
+ */
+sim_status sim_sweep_host(const sim_problem* problem, int32_t P, int32_t n_runs, const int32_t* variants,
+                          const int32_t* Ks, sim_delay delay, float eta, int32_t m, uint64_t seed,
+                          int32_t n_replicas, int64_t replica_base, const float* w0, int64_t iters,
+                          double* t, float* loss, float* dist2);
+
+/*
  * Clock-only simulation for callers that cannot allocate device memory.  (The paper has no
  * counterpart for this entry point: it exists for the sake of the library's users, not of the
  * method.)

@@ -21,7 +21,7 @@ STATUS = {0: "SIM_OK", 1: "SIM_ERR_ARG", 2: "SIM_ERR_ALLOC", 3: "SIM_ERR_CUDA", 
 
 EXPORTS = ["sim_create", "sim_set_params", "sim_set_adasync", "sim_set_tuning", "sim_reserve", "sim_run",
            "sim_trace_size", "sim_get_trace", "sim_get_params", "sim_n_params", "sim_last_error",
-           "sim_destroy", "sim_draw_delays", "sim_draw_indices", "sim_simulate_host", "sim_schedule_noalloc",
+           "sim_destroy", "sim_draw_delays", "sim_draw_indices", "sim_simulate_host", "sim_sweep_host", "sim_schedule_noalloc",
            "sim_noalloc_last_error"]
 
 
@@ -67,6 +67,8 @@ def _load():
     L.sim_draw_indices.argtypes = [u64, i64, i32, i32, i32, i64, i32, vp, vp]
     L.sim_simulate_host.argtypes = [C.POINTER(SimProblem), i32, i32, C.c_int, SimDelay, C.c_float, i32, u64,
                                     i32, i64, vp, i32, dbl, i64] + [vp] * 8
+    L.sim_sweep_host.argtypes = [C.POINTER(SimProblem), i32, i32, vp, vp, SimDelay, C.c_float, i32, u64, i32, i64, vp, i64,
+                                 vp, vp, vp]
     L.sim_schedule_noalloc.argtypes = [i32, i32, C.c_int, SimDelay, u64, i64, i32, i32, dbl, i64] + [vp] * 6
     L.sim_noalloc_last_error.argtypes = []
     L.sim_noalloc_last_error.restype = C.c_char_p
@@ -253,4 +255,38 @@ def simulate_host(data, *, P, K, variant, delay_kind, mu, shift=0.0, eta, m, see
     w0p = hp(w0, np.float32)
     _check(lib.sim_simulate_host(C.byref(prob), P, K, VARIANTS[variant], SimDelay(DELAYS[delay_kind], mu, shift),
                                  eta, m, seed, n_replicas, replica_base, w0p, K0, t_interval, iters, *ptrs))
+    return out
+
+
+def sweep_host(data, runs, *, P, delay_kind, mu, shift=0.0, eta, m, seed, n_replicas, iters, replica_base=0, w0=None,
+               w_ref=None, want=("t", "loss")):
+    """All (variant, K) pairs of `runs` on one HOST data set in one call: the data is copied in once,
+    the runs overlap on the device, the traces come back as [n_runs, R, iters] numpy arrays."""
+    model = data["model"]
+    prob = SimProblem(MODELS[model], 0, 0, 0, 0, None, None, None, None)
+    keep = []
+
+    def hp(a, dt):
+        if a is None:
+            return None
+        a = np.ascontiguousarray(a, dtype=dt)
+        keep.append(a)
+        return a.ctypes.data
+
+    prob.n, prob.d = data["X"].shape
+    prob.n_classes, prob.hidden = int(data.get("n_classes", 1)), int(data.get("hidden", 0))
+    prob.X = hp(data["X"], np.float32)
+    if model == "lsq":
+        prob.y = hp(data["y"], np.float32)
+    else:
+        prob.label = hp(data["y"], np.int32)
+    prob.w_ref = hp(w_ref, np.float32)
+    variants = np.array([VARIANTS[v] for v, _ in runs], np.int32)
+    Ks = np.array([k for _, k in runs], np.int32)
+    shape = (len(runs), n_replicas, iters)
+    out = {k: np.empty(shape, {"t": np.float64, "loss": np.float32, "dist2": np.float32}[k]) for k in want}
+    ptrs = [C.c_void_p(out[k].ctypes.data) if k in out else None for k in ("t", "loss", "dist2")]
+    _check(lib.sim_sweep_host(C.byref(prob), P, len(runs), C.c_void_p(variants.ctypes.data), C.c_void_p(Ks.ctypes.data),
+                              SimDelay(DELAYS[delay_kind], mu, shift), eta, m, seed, n_replicas, replica_base,
+                              hp(w0, np.float32), iters, *ptrs))
     return out

@@ -559,4 +559,70 @@ sim_status sim_simulate_host(const sim_problem* problem, int32_t P, int32_t K, s
   return SIM_OK;
 }
 
+sim_status sim_sweep_host(const sim_problem* problem, int32_t P, int32_t n_runs, const int32_t* variants,
+                          const int32_t* Ks, sim_delay delay, float eta, int32_t m, uint64_t seed,
+                          int32_t n_replicas, int64_t replica_base, const float* w0, int64_t iters,
+                          double* t, float* loss, float* dist2) {
+  if (!problem || problem->model == SIM_NONE || !problem->X) return fail(nullptr, SIM_ERR_ARG, "sim_sweep_host needs a problem");
+  if (n_runs < 1 || n_runs > 256 || !variants || !Ks) return fail(nullptr, SIM_ERR_ARG, "n_runs must be in [1, 256] with variants and Ks given");
+  if (iters < 1) return fail(nullptr, SIM_ERR_ARG, "iters must be >= 1");
+  if (problem->n < 1 || problem->d < 1) return fail(nullptr, SIM_ERR_ARG, "bad problem");
+  sim_problem dp = *problem;
+  const long long np = model_params(dp);
+  std::vector<void*> owned;
+  std::vector<sim_handle*> hs((size_t)n_runs, nullptr);
+  std::vector<cudaStream_t> streams((size_t)n_runs, nullptr);
+  sim_status st = SIM_OK;
+  std::string msg;
+  auto up = [&](const void* src, size_t bytes, void** dst) -> bool {
+    *dst = nullptr;
+    if (!src || bytes == 0) return true;
+    cudaError_t e = cudaMalloc(dst, bytes);
+    if (e == cudaSuccess) { owned.push_back(*dst); e = cudaMemcpyAsync(*dst, src, bytes, cudaMemcpyHostToDevice, nullptr); }
+    if (e != cudaSuccess) { st = e == cudaErrorMemoryAllocation ? SIM_ERR_ALLOC : SIM_ERR_CUDA; msg = cudaGetErrorString(e); return false; }
+    return true;
+  };
+  const size_t RJ = (size_t)n_replicas * (size_t)iters;
+  do {
+    void *X, *y, *lab, *wr, *dw0;
+    if (!up(problem->X, (size_t)dp.n * dp.d * 4, &X)) break;
+    if (!up(problem->y, (size_t)dp.n * 4, &y)) break;
+    if (!up(problem->label, (size_t)dp.n * 4, &lab)) break;
+    if (!up(problem->w_ref, (size_t)np * 4, &wr)) break;
+    if (!up(w0, (size_t)np * 4, &dw0)) break;
+    dp.X = (const float*)X; dp.y = (const float*)y; dp.label = (const int32_t*)lab; dp.w_ref = (const float*)wr;
+    if (cudaDeviceSynchronize() != cudaSuccess) { st = SIM_ERR_CUDA; msg = "upload failed"; break; }
+    // every run gets its own stream: the runs are independent and overlap on the device
+    for (int i = 0; i < n_runs && st == SIM_OK; ++i) {
+      if (cudaStreamCreateWithFlags(&streams[i], cudaStreamNonBlocking) != cudaSuccess) { st = SIM_ERR_CUDA; msg = "stream creation failed"; break; }
+      st = sim_create(&dp, P, Ks[i], (sim_variant)variants[i], delay, eta, m, seed, n_replicas, replica_base, streams[i], &hs[i]);
+      if (st != SIM_OK) { msg = g_last_error; break; }
+      if ((st = sim_reserve(hs[i], iters)) != SIM_OK) { msg = sim_last_error(hs[i]); break; }
+      if (dw0 && (st = sim_set_params(hs[i], (const float*)dw0)) != SIM_OK) { msg = sim_last_error(hs[i]); break; }
+    }
+    if (st != SIM_OK) break;
+    for (int i = 0; i < n_runs && st == SIM_OK; ++i)
+      if ((st = sim_run(hs[i], iters)) != SIM_OK) msg = sim_last_error(hs[i]);
+    if (st != SIM_OK) break;
+    // traces come back run by run, straight from each handle's buffers (row pitch = capacity = iters)
+    for (int i = 0; i < n_runs && st == SIM_OK; ++i) {
+      sim_handle* h = hs[i];
+      if ((st = device_error(h)) != SIM_OK) { msg = sim_last_error(h); break; }
+      cudaError_t e = cudaSuccess;
+      if (t) e = cudaMemcpy2D(t + (size_t)i * RJ, (size_t)iters * 8, h->tr.t, (size_t)h->cap * 8, (size_t)iters * 8, n_replicas, cudaMemcpyDeviceToHost);
+      if (e == cudaSuccess && loss) e = cudaMemcpy2D(loss + (size_t)i * RJ, (size_t)iters * 4, h->tr.loss, (size_t)h->cap * 4, (size_t)iters * 4, n_replicas, cudaMemcpyDeviceToHost);
+      if (e == cudaSuccess && dist2) e = cudaMemcpy2D(dist2 + (size_t)i * RJ, (size_t)iters * 4, h->tr.dist2, (size_t)h->cap * 4, (size_t)iters * 4, n_replicas, cudaMemcpyDeviceToHost);
+      if (e != cudaSuccess) { st = SIM_ERR_CUDA; msg = cudaGetErrorString(e); }
+    }
+  } while (0);
+  for (int i = 0; i < n_runs; ++i) {
+    if (hs[i]) sim_destroy(hs[i]);
+    if (streams[i]) cudaStreamDestroy(streams[i]);
+  }
+  cudaDeviceSynchronize();
+  for (void* p : owned) cudaFree(p);
+  if (st != SIM_OK) return fail(nullptr, st, "sim_sweep_host: " + msg);
+  return SIM_OK;
+}
+
 }  // extern "C"

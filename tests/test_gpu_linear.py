@@ -151,3 +151,18 @@ def test_host_buffer_call_matches_device_call(B):
         assert np.array_equal(out[k], tr[k]), k
     assert np.array_equal(out["w"], sim.params())
     sim.close()
+
+
+def test_sweep_on_host_buffers_matches_single_runs(B):
+    data = inputs.make_lsq(1500, 128, 0.1, 83)
+    runs = [("ksync", 1), ("ksync", 3), ("kbatchsync", 2), ("kbatchasync", 2)]
+    kw = dict(P=4, delay_kind="shifted_exp", mu=1.0, shift=0.5, eta=0.02, m=8, seed=5, n_replicas=6)
+    out = B.sweep_host(data, runs, iters=30, w_ref=data["w_star"], want=("t", "loss", "dist2"), **kw)
+    dev = to_device(data)
+    for i, (variant, K) in enumerate(runs):
+        sim = B.Simulation(dev, variant=variant, K=K, w_ref=torch.from_numpy(data["w_star"]).cuda(), **kw)
+        sim.run(30)
+        tr = sim.trace()
+        sim.close()
+        for k in ("t", "loss", "dist2"):
+            assert np.array_equal(out[k][i], tr[k]), (variant, K, k)
