@@ -35,6 +35,7 @@ struct MlpScratch {
   float* dW2_part = nullptr;       // [R][Kmax][H*C]
   float* db2_part = nullptr;       // [R][Kmax][16]
   float* loss_part = nullptr;      // [R][Kmax][m/32]
+  int* rows_tab = nullptr;         // [R][Kmax][m]             sample row of every minibatch draw of the current update
   int H = 0, C = 0, d = 0, m = 0, Kmax = 0, n_slots = 0, R = 0;
   long long n = 0;
 };
@@ -88,6 +89,22 @@ __global__ void shadow_w1_kernel(const float* pool, __nv_bfloat16* W1qT, long lo
     const long long r = i / dH, p = i % dH;
     const long long n = p / d, k = p % d;       // output element (n, k) = W1[k][n]
     W1qT[((size_t)r * n_slots + slot) * dH + p] = __float2bfloat16_rn(pool[((size_t)r * n_slots + slot) * slot_stride + k * H + n]);
+  }
+}
+
+// ---- sample rows of the update's minibatches, drawn once for all kernels of the update ----------
+__global__ void mlp_rows_kernel(MlpArgs g) {
+  const NumericArgs& a = g.na;
+  const MlpScratch& sc = g.sc;
+  const int l = blockIdx.x % sc.Kmax, r = blockIdx.x / sc.Kmax;
+  const int K = (int)a.K_used[(size_t)r * a.cap + g.j];
+  if (l >= K) return;
+  const size_t ent = ((size_t)r * a.cap + g.j) * a.K_stride + l;
+  const uint32_t worker = a.worker[ent], seq = a.seq[ent];
+  for (int q = threadIdx.x; q < sc.m; q += blockDim.x) {
+    uint32_t idx = draw_index(a.seed, a.replica_base + (uint32_t)r, worker, seq, (uint32_t)q, a.n);
+    if ((uint64_t)idx >= a.n) { atomicExch(a.err, ERR_BAD_INDEX); idx = 0; }
+    sc.rows_tab[((size_t)r * sc.Kmax + l) * sc.m + q] = (int)idx;
   }
 }
 
@@ -161,7 +178,7 @@ __global__ void __launch_bounds__(256) mlp_small_update_kernel(MlpArgs g) {
 
 // ---- host side -----------------------------------------------------------------------------------
 inline void mlp_scratch_free(MlpScratch& s) {
-  cudaFree(s.Xq); cudaFree(s.W1qT); cudaFree(s.D1q); cudaFree(s.Hact); cudaFree(s.D2);
+  cudaFree(s.rows_tab); cudaFree(s.Xq); cudaFree(s.W1qT); cudaFree(s.D1q); cudaFree(s.Hact); cudaFree(s.D2);
   cudaFree(s.db1_part); cudaFree(s.dW2_part); cudaFree(s.db2_part); cudaFree(s.loss_part);
   s = MlpScratch{};
 }
@@ -183,6 +200,7 @@ inline cudaError_t mlp_scratch_alloc(MlpScratch& s, const float* X, long long n,
   MLP_ALLOC(s.dW2_part, tasks * H * C)
   MLP_ALLOC(s.db2_part, tasks * 16)
   MLP_ALLOC(s.loss_part, tasks * (m / 32))
+  MLP_ALLOC(s.rows_tab, tasks * m)
 #undef MLP_ALLOC
   to_bf16_kernel<<<1184, 256, 0, stream>>>(X, s.Xq, (long long)n * d);
   return cudaGetLastError();

@@ -350,177 +350,202 @@ __device__ __forceinline__ uint64_t tc_desc_mnmajor(uint32_t saddr, uint32_t lbo
          ((uint64_t)2 << 61);
 }
 
-struct TcDw1Layout { int stages, stage_bytes, off_rows, off_bars, off_tmem, total; };
-// columns of W1 handled by one CTA of the dW1 kernel: 128 where H allows, so that three CTAs
-// (128 tensor-memory columns and ~70 KB of shared memory each) share an SM and one CTA's
-// row-per-thread epilogue overlaps the others' loads
-inline __host__ __device__ int tc_dw1_cols(int H) { return H % 128 == 0 ? 128 : 64; }
-inline __host__ __device__ TcDw1Layout tc_dw1_layout(int H, int max_samples) {
+// ---- dW1 = bf16(X)^T bf16(delta1), fused with the update of W1: persistent kernel -----------------
+// Tiles of 128 rows of W1 x Hn columns (Hn <= 256) are dealt round-robin to one CTA per SM.  The
+// accumulator is double-buffered in tensor memory, so the row-per-thread epilogue of one tile
+// (read w_j, apply Eq. 2 / Eq. 3, write w_{j+1} and its transposed bf16 shadow) overlaps the loads
+// and MMAs of the next.  Both operands are MN-major and used exactly as stored: a stage holds 64
+// samples; A = their features [slab*128, +128) gathered from the bf16 data set (cp.async by four
+// producer warps into the 128-byte-swizzle atom layout), B = the same samples' bf16 delta1 columns
+// (TMA boxes of 64 x 64).  dW1 itself never exists in memory.
+//   warp 0      TMA producer of B          warp 1      tcgen05.mma issuer, owns tensor memory
+//   warps 2-5   cp.async producers of A    warps 6-13  epilogue (one row of W1 per thread, two warps per
+//                                                      tensor-memory lane quarter, half of the columns each)
+constexpr int DW1_THREADS = 448;
+
+// columns per tile: the largest H/p that is at most 256 and a multiple of 64
+inline __host__ __device__ int tc_dw1_cols(int H) {
+  for (int p = 1; p <= 8; ++p)
+    if (H % p == 0 && H / p <= 256 && (H / p) % 64 == 0) return H / p;
+  return 64;
+}
+struct TcDw1Layout { int stages, stage_bytes, off_bars, off_tmem, total; };
+inline __host__ __device__ TcDw1Layout tc_dw1_layout(int H) {
   TcDw1Layout L;
-  const int Hc = tc_dw1_cols(H);
-  L.stage_bytes = TC_A_BYTES + Hc * 128;      // A: 64 samples x 128 features; B: 64 samples x Hc
-  L.stages = 2;
-  L.off_rows = L.stages * L.stage_bytes;
-  L.off_bars = L.off_rows + max_samples * 4;
-  L.off_tmem = L.off_bars + 8 * (2 * L.stages + 1);
+  L.stage_bytes = TC_A_BYTES + tc_dw1_cols(H) * 128;     // A: 64 samples x 128 features; B: 64 samples x Hn
+  L.stages = (200 << 10) / L.stage_bytes;
+  if (L.stages > 4) L.stages = 4;
+  L.off_bars = L.stages * L.stage_bytes;
+  L.off_tmem = L.off_bars + 8 * (2 * L.stages + 4);
   L.total = L.off_tmem + 16 + 1024;
   return L;
 }
 
-// dW1 = bf16(X)^T bf16(delta1) over all K m samples of the update, fused with the update of W1.
-// One CTA per (replica, 128-row slab of W1, block of Hc columns); the 128 x Hc accumulator lives in
-// tensor memory.
-// Both operands are MN-major: a stage holds 64 samples; A = their features [slab*128, +128) as
-// gathered from the bf16 data set (cp.async by warps 2-5, written in the swizzled atom layout),
-// B = the same samples' bf16 delta1 rows (TMA boxes of 64 x 64).  The epilogue applies
-// W1 <- W1 - (eta/(K m)) dW1 (Eq. 2 / Eq. 3) and writes the new fp32 version and its transposed
-// bf16 shadow; dW1 itself never exists in memory.
-__global__ void __launch_bounds__(TC_THREADS)
+__global__ void __launch_bounds__(DW1_THREADS, 1)
 mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
   const NumericArgs& a = g.na;
   const MlpScratch& sc = g.sc;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int H = sc.H, d = sc.d, m = sc.m;
-  const int slabs = d / 128;
-  const int Hc = tc_dw1_cols(H), splits = H / Hc;
-  const int cs = blockIdx.x % splits;                 // column block
-  const int slab = (blockIdx.x / splits) % slabs, r = blockIdx.x / (splits * slabs);
-  const int col0 = cs * Hc;
+  const int slabs = d / 128, Hn = tc_dw1_cols(H), parts = H / Hn;
+  const int n_tiles = a.R * slabs * parts;
   const long long j = g.j;
-  const int K = (int)a.K_used[(size_t)r * a.cap + j];
-  const uint32_t rid = a.replica_base + (uint32_t)r;
   const long long dH = (long long)d * H;
   const int blocks_per_task = m / TC_BK;
-  const int nk = K * blocks_per_task;
-  const int n_inst = Hc;                              // <= 128: one MMA covers the CTA's columns
   uint32_t tmem_cols = 32;
-  while ((int)tmem_cols < Hc) tmem_cols <<= 1;
+  while ((int)tmem_cols < 2 * Hn) tmem_cols <<= 1;
 
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw_addr = smem_addr(smem_raw);
   const uint32_t base_addr = (raw_addr + 1023u) & ~1023u;
   unsigned char* base = smem_raw + (base_addr - raw_addr);
-  const TcDw1Layout L = tc_dw1_layout(H, sc.Kmax * m);
+  const TcDw1Layout L = tc_dw1_layout(H);
   const int S = L.stages;
-  int* rows_s = reinterpret_cast<int*>(base + L.off_rows);
-  const uint32_t bars = base_addr + L.off_bars;
+  const uint32_t bars = base_addr + L.off_bars;     // full[S] | empty[S] | acc_full[2] | acc_empty[2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base + L.off_tmem);
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (S + s); };
-  const uint32_t acc_bar = bars + 8u * (2 * S);
+  auto acc_full = [&](int b) { return bars + 8u * (2 * S + b); };
+  auto acc_empty = [&](int b) { return bars + 8u * (2 * S + 2 + b); };
 
   if (tid == 0) {
     for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1 + 128); mbar_init(empty_bar(s), 1); }
-    mbar_init(acc_bar, 1);
+    for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 8); }
     mbar_fence_init();
   }
   if (warp == 1) tc_alloc(smem_addr(tmem_slot), tmem_cols);
-  for (int i = tid; i < K * m; i += TC_THREADS) {      // sample rows of the whole update, contributor-major
-    const int l = i / m, q = i % m;
-    const size_t ent = ((size_t)r * a.cap + j) * a.K_stride + l;
-    uint32_t idx = draw_index(a.seed, rid, a.worker[ent], a.seq[ent], (uint32_t)q, a.n);
-    if ((uint64_t)idx >= a.n) { atomicExch(a.err, ERR_BAD_INDEX); idx = 0; }
-    rows_s[i] = (int)idx;
-  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   bool failed = false;
   const uint32_t ATOM = 8192;     // one 64-wide MN block of a 64-sample stage: 64 k-rows x 128 B
+  // tile t -> (replica, slab, column part); the number of 64-sample stages depends on the replica's K
+  auto tile_r = [&](int t) { return t / (parts * slabs); };
+  auto tile_nk = [&](int t) { return (int)a.K_used[(size_t)tile_r(t) * a.cap + j] * blocks_per_task; };
 
   if (warp == 0) {
-    // ---- B producer: delta1 rows of 64 samples, H/64 boxes of 64 x 64 ----
+    // ---- B producer: delta1 rows of 64 samples, Hn/64 boxes of 64 x 64 ----
     if (lane == 0) {
-      for (int kc = 0; kc < nk; ++kc) {
-        const int s = kc % S;
-        if (!mbar_wait(empty_bar(s), (uint32_t)(((kc / S) & 1) ^ 1))) { failed = true; break; }
-        const uint32_t Bs = base_addr + (uint32_t)s * L.stage_bytes + TC_A_BYTES;
-        const int l = kc / blocks_per_task, blk = kc % blocks_per_task;
-        const int row0 = (int)(((size_t)r * sc.Kmax + l) * m + (size_t)blk * TC_BK);
-        mbar_arrive_expect_tx(full_bar(s), (uint32_t)(Hc * 128));
-        for (int b = 0; b < Hc / 64; ++b) tma_load_2d(Bs + (uint32_t)b * ATOM, &tmD, col0 + b * 64, row0, full_bar(s));
+      long long it = 0;
+      for (int t = blockIdx.x; t < n_tiles && !failed; t += gridDim.x) {
+        const int r = tile_r(t), part = t % parts, nk = tile_nk(t);
+        for (int kc = 0; kc < nk; ++kc, ++it) {
+          const int s = (int)(it % S);
+          if (!mbar_wait(empty_bar(s), (uint32_t)(((it / S) & 1) ^ 1))) { failed = true; break; }
+          const uint32_t Bs = base_addr + (uint32_t)s * L.stage_bytes + TC_A_BYTES;
+          const int row0 = (int)((size_t)r * sc.Kmax * m + (size_t)kc * TC_BK);
+          mbar_arrive_expect_tx(full_bar(s), (uint32_t)(Hn * 128));
+          for (int b = 0; b < Hn / 64; ++b) tma_load_2d(Bs + (uint32_t)b * ATOM, &tmD, part * Hn + b * 64, row0, full_bar(s));
+        }
       }
     }
     __syncwarp();
   } else if (warp == 1) {
     // ---- MMA issuer ----
-    const uint32_t idesc = tc_idesc(n_inst, 1, 1);
+    const uint32_t idesc = tc_idesc(Hn, 1, 1);
     const uint32_t lbo = ATOM, sbo = 1024u;   // next 64 MN elements: one atom block on; next 8 samples: 1024 B on
-    for (int kc = 0; kc < nk; ++kc) {
-      const int s = kc % S;
-      if (!mbar_wait(full_bar(s), (uint32_t)((kc / S) & 1))) { failed = true; break; }
+    long long it = 0;
+    int i = 0;
+    for (int t = blockIdx.x; t < n_tiles && !failed; t += gridDim.x, ++i) {
+      const int nk = tile_nk(t), buf = i & 1;
+      if (!mbar_wait(acc_empty(buf), (uint32_t)(((i >> 1) & 1) ^ 1))) { failed = true; break; }
       tc_fence_after();
-      if (lane == 0) {
-        const uint32_t As = base_addr + (uint32_t)s * L.stage_bytes, Bs = As + TC_A_BYTES;
+      for (int kc = 0; kc < nk; ++kc, ++it) {
+        const int s = (int)(it % S);
+        if (!mbar_wait(full_bar(s), (uint32_t)((it / S) & 1))) { failed = true; break; }
+        tc_fence_after();
+        if (lane == 0) {
+          const uint32_t As = base_addr + (uint32_t)s * L.stage_bytes, Bs = As + TC_A_BYTES;
 #pragma unroll
-        for (int k16 = 0; k16 < TC_BK / 16; ++k16) {      // 16 samples = two 8-row groups = 2048 B
-          const uint64_t ad = tc_desc_mnmajor(As + k16 * 2048, lbo, sbo);
-          const uint64_t bd = tc_desc_mnmajor(Bs + k16 * 2048, lbo, sbo);
-          tc_mma_bf16(tmem_base, ad, bd, idesc, (kc > 0 || k16 > 0) ? 1u : 0u);
+          for (int k16 = 0; k16 < TC_BK / 16; ++k16) {      // 16 samples = two 8-row groups = 2048 B
+            const uint64_t ad = tc_desc_mnmajor(As + k16 * 2048, lbo, sbo);
+            const uint64_t bd = tc_desc_mnmajor(Bs + k16 * 2048, lbo, sbo);
+            tc_mma_bf16(tmem_base + (uint32_t)buf * Hn, ad, bd, idesc, (kc > 0 || k16 > 0) ? 1u : 0u);
+          }
+          tc_commit(empty_bar(s));
+          if (kc == nk - 1) tc_commit(acc_full(buf));
         }
-        tc_commit(empty_bar(s));
-        if (kc == nk - 1) tc_commit(acc_bar);
+        __syncwarp();
       }
-      __syncwarp();
     }
-  } else {
-    // The CTA's whole working set is known now: ask L2 for it at once (the 256-byte feature slices
-    // of all K m sample rows and this thread's row of w_j), so that the short software pipeline
-    // below runs against L2 latency instead of one DRAM round trip per stage.
-    {
-      const int t = tid - 64;
-      for (int i = t; i < 2 * K * m; i += 128)
-        prefetch_l2(sc.Xq + (size_t)rows_s[i >> 1] * d + (size_t)slab * 128 + (i & 1) * 64);
-      const float* wrow = a.pool + ((size_t)r * a.n_slots + mlp_cur_slot(a, r, j)) * a.slot_stride +
-                          ((size_t)slab * 128 + 32 * (warp & 3) + lane) * H + col0;
-      for (int i = 0; i < Hc / 32; ++i) prefetch_l2(wrow + i * 32);
-    }
-    // ---- A producer: thread t copies 16-byte piece (t & 15) of sample rows (t >> 4) + 8 i, i < 8 ----
-    {
-      const int t = tid - 64, piece = t & 15, k0 = t >> 4;
-      auto signal = [&](int kc2) {
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        mbar_arrive(full_bar(kc2 % S));
-      };
-      int signalled = 0;
-      for (int kc = 0; kc < nk && !failed; ++kc) {
-        const int s = kc % S;
-        if (!mbar_wait(empty_bar(s), (uint32_t)(((kc / S) & 1) ^ 1))) { failed = true; break; }
+  } else if (warp < 6) {
+    // ---- A producers: thread p copies 16-byte piece (p & 15) of sample rows (p >> 4) + 8 i, i < 8 ----
+    const int p = tid - 64, piece = p & 15, k0 = p >> 4;
+    long long it = 0, signalled = 0;
+    auto signal = [&](long long which) {
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      mbar_arrive(full_bar((int)(which % S)));
+    };
+    for (int t = blockIdx.x; t < n_tiles && !failed; t += gridDim.x) {
+      const int r = tile_r(t), slab = (t / parts) % slabs, nk = tile_nk(t);
+      const int* rows = sc.rows_tab + (size_t)r * sc.Kmax * m;
+      for (int kc = 0; kc < nk; ++kc, ++it) {
+        const int s = (int)(it % S);
+        int rid[8];                     // issued before the wait: the ring is usually full, the latency hides there
+#pragma unroll
+        for (int i = 0; i < 8; ++i) rid[i] = rows[kc * TC_BK + k0 + 8 * i];
+        if (!mbar_wait(empty_bar(s), (uint32_t)(((it / S) & 1) ^ 1))) { failed = true; break; }
         const uint32_t As = base_addr + (uint32_t)s * L.stage_bytes + (uint32_t)(piece >> 3) * ATOM;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const int k = k0 + 8 * i;
           cp_async16(As + (k >> 3) * 1024 + (k & 7) * 128 + (((piece & 7) ^ (k & 7)) << 4),
-                     sc.Xq + (size_t)rows_s[kc * TC_BK + k] * d + (size_t)slab * 128 + piece * 8);
+                     sc.Xq + (size_t)rid[i] * d + (size_t)slab * 128 + piece * 8);
         }
         cp_async_commit();
-        if (kc >= S - 1) {
-          if (S == 2) cp_async_wait<1>(); else cp_async_wait<3>();
+        if (it >= S - 1) {              // the group issued S-1 stages ago has landed
+          if (S == 2) cp_async_wait<1>(); else if (S == 3) cp_async_wait<2>(); else cp_async_wait<3>();
           signal(signalled++);
         }
       }
-      cp_async_wait<0>();
-      if (!failed) while (signalled < nk) signal(signalled++);
     }
-    // ---- epilogue: thread = one row of W1 ----
-    const int q = warp & 3;
-    const size_t row = (size_t)slab * 128 + 32 * q + lane;
-    if (!failed && !mbar_wait(acc_bar, 0)) failed = true;
-    tc_fence_after();
-    if (!failed) {
-      const uint32_t trow = tmem_base + ((uint32_t)(32 * q) << 16);
-      const int cur = mlp_cur_slot(a, r, j), fresh = mlp_fresh_slot(a, r, j);
+    cp_async_wait<0>();
+    if (!failed) while (signalled < it) signal(signalled++);
+  } else {
+    // ---- epilogue: thread = one row of W1 of the tile, columns [half*Hn/2, +Hn/2) ----
+    const int q = warp & 3;             // the tensor-memory lane quarter this warp may read
+    const int half = (warp - 6) >> 2, Hh = Hn / 2, nch = Hh / 32;
+    auto tile_ptr = [&](int t) {        // this thread's part of w_j in tile t
+      const int r = tile_r(t), slab = (t / parts) % slabs, part = t % parts;
+      return a.pool + ((size_t)r * a.n_slots + mlp_cur_slot(a, r, j)) * a.slot_stride +
+             ((size_t)slab * 128 + 32 * q + lane) * H + part * Hn + half * Hh;
+    };
+    int i = 0;
+    if ((int)blockIdx.x < n_tiles) { const float* p0 = tile_ptr(blockIdx.x); for (int c = 0; c < nch; ++c) prefetch_l2(p0 + c * 32); }
+    for (int t = blockIdx.x; t < n_tiles && !failed; t += gridDim.x, ++i) {
+      const int r = tile_r(t), slab = (t / parts) % slabs, part = t % parts, buf = i & 1;
+      const int K = (int)a.K_used[(size_t)r * a.cap + j];
+      const size_t row = (size_t)slab * 128 + 32 * q + lane;
+      const int col0 = part * Hn + half * Hh;
+      const int fresh = mlp_fresh_slot(a, r, j);
       const float scale = (float)((double)a.eta / ((double)K * (double)m));
-      const float* wc = a.pool + ((size_t)r * a.n_slots + cur) * a.slot_stride + row * H + col0;
+      const float* wc = tile_ptr(t);
       float* wn = a.pool + ((size_t)r * a.n_slots + fresh) * a.slot_stride + row * H + col0;
-      __nv_bfloat16* wq = sc.W1qT + ((size_t)r * sc.n_slots + fresh) * dH + (size_t)col0 * d + row;   // [H][d], this row's column
+      __nv_bfloat16* wq = sc.W1qT + ((size_t)r * sc.n_slots + fresh) * dH + (size_t)col0 * d + row;   // [H][d]
+      if (t + (int)gridDim.x < n_tiles) {            // the next tile's w_j: ask L2 for it a whole tile ahead
+        const float* pn = tile_ptr(t + gridDim.x);
+        for (int c = 0; c < nch; ++c) prefetch_l2(pn + c * 32);
+      }
+      float4 wnext[8];                                // w_j of the chunk after the one being processed
+#pragma unroll
+      for (int i4 = 0; i4 < 8; ++i4) wnext[i4] = reinterpret_cast<const float4*>(wc)[i4];
+      if (!mbar_wait(acc_full(buf), (uint32_t)((i >> 1) & 1))) { failed = true; break; }
+      tc_fence_after();
+      const uint32_t trow = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * Hn + half * Hh);
       uint32_t v[32];
-      for (int ch = 0; ch < Hc / 32; ++ch) {
+      for (int ch = 0; ch < nch; ++ch) {
+        float4 wcur[8];
+#pragma unroll
+        for (int i4 = 0; i4 < 8; ++i4) wcur[i4] = wnext[i4];
+        if (ch + 1 < nch) {
+#pragma unroll
+          for (int i4 = 0; i4 < 8; ++i4) wnext[i4] = reinterpret_cast<const float4*>(wc + (ch + 1) * 32)[i4];
+        }
         tc_ld32(trow + ch * 32, v);
 #pragma unroll
         for (int i4 = 0; i4 < 8; ++i4) {
-          float4 w = reinterpret_cast<const float4*>(wc + ch * 32)[i4];
+          float4 w = wcur[i4];
           w.x = fmaf(-scale, __uint_as_float(v[4 * i4]), w.x);
           w.y = fmaf(-scale, __uint_as_float(v[4 * i4 + 1]), w.y);
           w.z = fmaf(-scale, __uint_as_float(v[4 * i4 + 2]), w.z);
@@ -533,6 +558,9 @@ mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
           wq[(size_t)(col + 3) * d] = __float2bfloat16_rn(w.w);
         }
       }
+      tc_fence_before();                 // this warp's reads of the buffer are done: hand it back
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty(buf));
     }
   }
 
@@ -587,17 +615,22 @@ inline cudaError_t run_mlp(NumericArgs& a, MlpScratch& s, MlpMaps& maps, int P, 
   }
   const TcLayout L = tc_forward_layout(s.H);
   if ((e = cudaFuncSetAttribute(mlp_forward_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total)) != cudaSuccess) return e;
-  const TcDw1Layout LD = tc_dw1_layout(s.H, s.Kmax * s.m);
-  if (LD.total > (227 << 10)) { *why = "mlp: K_max * m too large for the dW1 kernel's row table"; return cudaSuccess; }
+  const TcDw1Layout LD = tc_dw1_layout(s.H);
   if ((e = cudaFuncSetAttribute(mlp_dw1_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, LD.total)) != cudaSuccess) return e;
+  int dev = 0, sms = 148;
+  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+  if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+  const int dw1_tiles = a.R * (s.d / 128) * (s.H / tc_dw1_cols(s.H));
+  const int dw1_grid = dw1_tiles < sms ? dw1_tiles : sms;      // one persistent CTA per SM
   MlpArgs g{};
   g.na = a; g.sc = s; g.H = s.H; g.P = P;
   const int mtiles = s.m / 128;
   for (long long u = 0; u < a.iters; ++u) {
     g.j = a.j0 + u;
+    mlp_rows_kernel<<<a.R * s.Kmax, 128, 0, stream>>>(g);
     mlp_forward_tc_kernel<<<a.R * s.Kmax * mtiles, TC_THREADS, L.total, stream>>>(maps.tmX, maps.tmW, g);
     mlp_head_kernel<<<a.R * s.Kmax, 512, (size_t)s.m * 16 * 4, stream>>>(g);
-    mlp_dw1_tc_kernel<<<a.R * (s.d / 128) * (s.H / tc_dw1_cols(s.H)), TC_THREADS, LD.total, stream>>>(maps.tmD, g);
+    mlp_dw1_tc_kernel<<<dw1_grid, DW1_THREADS, LD.total, stream>>>(maps.tmD, g);
     mlp_small_update_kernel<<<a.R, 256, 0, stream>>>(g);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
