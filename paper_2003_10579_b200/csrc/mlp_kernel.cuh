@@ -8,16 +8,17 @@
 //     dW1 = bf16(X_b)^T bf16(delta1)   (backward, [d x m] [m x H])
 // everything else (bias, relu, layer 2, softmax, loss, update) is fp32.
 //
-// All replicas advance in lock step, one update at a time, with four launches per update:
+// All replicas advance in lock step, one update at a time, with four launches per update (rows,
+// forward, head, dw1):
 //   forward   (mlp_tc_kernel.cuh) one CTA per (replica, contributor, 128-sample block): A1 = X_b W1 on
 //             tcgen05 with the accumulator in tensor memory, then h = relu(A1 + b1), logits, softmax,
 //             delta2, delta1 = (delta2 W2^T) . [h > 0]; writes h, delta2, bf16(delta1), partial db1, loss
-//   head      one CTA per (replica, contributor): dW2 = h^T delta2, db2
+//   head      one CTA per (replica, contributor): dW2 = h^T delta2, db2; the replica's last CTA then
+//             updates b1, W2, b2 from the partials (fixed summation order) and records the loss
 //   dw1       (mlp_tc_kernel.cuh) one CTA per (replica, 128-row slab of W1): accumulates X^T delta1 over
 //             all K m samples of the update in tensor memory (tcgen05, MN-major operands) and applies
 //             W1 <- W1 - (eta/(K m)) dW1 in its epilogue (Eq. 2 / Eq. 3), writing the new version and
 //             its transposed bf16 shadow: dW1 never exists in memory
-//   small     b1, W2, b2 update from the partials (fixed summation order), loss record
 #pragma once
 #include <cuda_bf16.h>
 
@@ -35,6 +36,7 @@ struct MlpScratch {
   float* dW2_part = nullptr;       // [R][Kmax][H*C]
   float* db2_part = nullptr;       // [R][Kmax][16]
   float* loss_part = nullptr;      // [R][Kmax][m/32]
+  int* done_cnt = nullptr;         // [R]                      contributors whose head partials are complete
   int* rows_tab = nullptr;         // [R][Kmax][m]             sample row of every minibatch draw of the current update
   int H = 0, C = 0, d = 0, m = 0, Kmax = 0, n_slots = 0, R = 0;
   long long n = 0;
@@ -108,6 +110,39 @@ __global__ void mlp_rows_kernel(MlpArgs g) {
   }
 }
 
+// ---- b1, W2, b2 update and the loss record -------------------------------------------------------
+// (run by the last head CTA of a replica to finish: fixed summation order over contributors)
+__device__ void mlp_small_update(const MlpArgs& g, int r, int tid, int nthreads) {
+  const NumericArgs& a = g.na;
+  const MlpScratch& sc = g.sc;
+  const long long j = g.j;
+  const int K = (int)a.K_used[(size_t)r * a.cap + j];
+  const int H = sc.H, C = sc.C, m = sc.m, halves = m / 32;   // partial sums per 32-row group
+  const long long dH = (long long)sc.d * H;
+  const int cur = mlp_cur_slot(a, r, j), fresh = mlp_fresh_slot(a, r, j);
+  const float scale = (float)((double)a.eta / ((double)K * (double)m));
+  const float* wc = a.pool + ((size_t)r * a.n_slots + cur) * a.slot_stride + dH;
+  float* wn = a.pool + ((size_t)r * a.n_slots + fresh) * a.slot_stride + dH;
+  const int tail = H + H * C + C;
+  for (int p = tid; p < tail; p += nthreads) {
+    float gsum = 0.f;
+    for (int l = 0; l < K; ++l) {
+      const size_t task = (size_t)r * sc.Kmax + l;
+      if (p < H) { for (int hf = 0; hf < halves; ++hf) gsum += sc.db1_part[(task * halves + hf) * H + p]; }
+      else if (p < H + H * C) gsum += sc.dW2_part[task * H * C + (p - H)];
+      else gsum += sc.db2_part[task * 16 + (p - H - H * C)];
+    }
+    wn[p] = fmaf(-scale, gsum, wc[p]);
+  }
+  if (tid == 0) {
+    float ls = 0.f;
+    for (int l = 0; l < K; ++l)
+      for (int hf = 0; hf < halves; ++hf) ls += sc.loss_part[((size_t)r * sc.Kmax + l) * halves + hf];
+    a.loss[(size_t)r * a.cap + j] = ls / ((float)K * (float)m);
+    a.dist2[(size_t)r * a.cap + j] = 0.f;
+  }
+}
+
 // ---- dW2 = h^T delta2, db2 (per contributor) --------------------------------------------------
 __global__ void __launch_bounds__(512) mlp_head_kernel(MlpArgs g) {
   const NumericArgs& a = g.na;
@@ -141,44 +176,22 @@ __global__ void __launch_bounds__(512) mlp_head_kernel(MlpArgs g) {
     for (int row = 0; row < m; ++row) s += d2_s[row * 16 + tid];
     sc.db2_part[task * 16 + tid] = s;
   }
-}
-
-// ---- b1, W2, b2 update and the loss record -------------------------------------------------------
-__global__ void __launch_bounds__(256) mlp_small_update_kernel(MlpArgs g) {
-  const NumericArgs& a = g.na;
-  const MlpScratch& sc = g.sc;
-  const int r = blockIdx.x, tid = threadIdx.x;
-  const long long j = g.j;
-  const int K = (int)a.K_used[(size_t)r * a.cap + j];
-  const int H = sc.H, C = sc.C, m = sc.m, halves = m / 32;   // partial sums per 32-row group
-  const long long dH = (long long)sc.d * H;
-  const int cur = mlp_cur_slot(a, r, j), fresh = mlp_fresh_slot(a, r, j);
-  const float scale = (float)((double)a.eta / ((double)K * (double)m));
-  const float* wc = a.pool + ((size_t)r * a.n_slots + cur) * a.slot_stride + dH;
-  float* wn = a.pool + ((size_t)r * a.n_slots + fresh) * a.slot_stride + dH;
-  const int tail = H + H * C + C;
-  for (int p = tid; p < tail; p += blockDim.x) {
-    float gsum = 0.f;
-    for (int l = 0; l < K; ++l) {
-      const size_t task = (size_t)r * sc.Kmax + l;
-      if (p < H) { for (int hf = 0; hf < halves; ++hf) gsum += sc.db1_part[(task * halves + hf) * H + p]; }
-      else if (p < H + H * C) gsum += sc.dW2_part[task * H * C + (p - H)];
-      else gsum += sc.db2_part[task * 16 + (p - H - H * C)];
-    }
-    wn[p] = fmaf(-scale, gsum, wc[p]);
-  }
-  if (tid == 0) {
-    float ls = 0.f;
-    for (int l = 0; l < K; ++l)
-      for (int hf = 0; hf < halves; ++hf) ls += sc.loss_part[((size_t)r * sc.Kmax + l) * halves + hf];
-    a.loss[(size_t)r * a.cap + j] = ls / ((float)K * (float)m);
-    a.dist2[(size_t)r * a.cap + j] = 0.f;
+  // the last of the replica's K contributor CTAs to get here applies the b1 / W2 / b2 update
+  __shared__ int is_last;
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) is_last = atomicAdd(&sc.done_cnt[r], 1) == K - 1;
+  __syncthreads();
+  if (is_last) {
+    __threadfence();
+    mlp_small_update(g, r, tid, blockDim.x);
+    if (tid == 0) sc.done_cnt[r] = 0;
   }
 }
 
 // ---- host side -----------------------------------------------------------------------------------
 inline void mlp_scratch_free(MlpScratch& s) {
-  cudaFree(s.rows_tab); cudaFree(s.Xq); cudaFree(s.W1qT); cudaFree(s.D1q); cudaFree(s.Hact); cudaFree(s.D2);
+  cudaFree(s.done_cnt); cudaFree(s.rows_tab); cudaFree(s.Xq); cudaFree(s.W1qT); cudaFree(s.D1q); cudaFree(s.Hact); cudaFree(s.D2);
   cudaFree(s.db1_part); cudaFree(s.dW2_part); cudaFree(s.db2_part); cudaFree(s.loss_part);
   s = MlpScratch{};
 }
@@ -201,6 +214,7 @@ inline cudaError_t mlp_scratch_alloc(MlpScratch& s, const float* X, long long n,
   MLP_ALLOC(s.db2_part, tasks * 16)
   MLP_ALLOC(s.loss_part, tasks * (m / 32))
   MLP_ALLOC(s.rows_tab, tasks * m)
+  MLP_ALLOC(s.done_cnt, (size_t)R)
 #undef MLP_ALLOC
   to_bf16_kernel<<<1184, 256, 0, stream>>>(X, s.Xq, (long long)n * d);
   return cudaGetLastError();

@@ -631,7 +631,6 @@ inline cudaError_t run_mlp(NumericArgs& a, MlpScratch& s, MlpMaps& maps, int P, 
     mlp_forward_tc_kernel<<<a.R * s.Kmax * mtiles, TC_THREADS, L.total, stream>>>(maps.tmX, maps.tmW, g);
     mlp_head_kernel<<<a.R * s.Kmax, 512, (size_t)s.m * 16 * 4, stream>>>(g);
     mlp_dw1_tc_kernel<<<dw1_grid, DW1_THREADS, LD.total, stream>>>(maps.tmD, g);
-    mlp_small_update_kernel<<<a.R, 256, 0, stream>>>(g);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
   return cudaSuccess;
