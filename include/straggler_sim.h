@@ -65,8 +65,10 @@ typedef enum {
 } sim_model;
 
 /* Per-minibatch compute time X of a worker, i.i.d. over workers and minibatches (Section 3.1):
- * X = Exp(mu) (rate mu, mean 1/mu) or shift + Exp(mu) (Lemma 4's shifted exponential). */
-typedef enum { SIM_DELAY_EXP = 0, SIM_DELAY_SHIFTED_EXP = 1 } sim_delay_kind;
+ * X = Exp(mu) (rate mu, mean 1/mu), shift + Exp(mu) (Lemma 4's shifted exponential), or the
+ * heavy-tailed Pareto law of the runtime simulations of Section 3 (Figs. 4-5) with shape mu = 2
+ * (the only shape built) and scale shift > 0: P(X > x) = (shift / x)^2. */
+typedef enum { SIM_DELAY_EXP = 0, SIM_DELAY_SHIFTED_EXP = 1, SIM_DELAY_PARETO2 = 2 } sim_delay_kind;
 typedef struct { sim_delay_kind kind; double mu; double shift; } sim_delay;
 
 /* The data set S of N samples (Section 2).  All pointers are DEVICE pointers, borrowed. */

@@ -17,7 +17,7 @@ _SRC = os.path.join(_HERE, "sched_core.c")
 _LIB = os.path.join(_HERE, "liboracle_core.so")
 
 VARIANTS = {"ksync": 0, "kbatchsync": 1, "kasync": 2, "kbatchasync": 3}
-DELAYS = {"exp": 0, "shifted_exp": 1}
+DELAYS = {"exp": 0, "shifted_exp": 1, "pareto2": 2}
 
 
 def build(force: bool = False) -> str:
@@ -83,7 +83,8 @@ def neg_log_uniform(x0: int, x1: int) -> float:
 
 
 def delay(kind: str, mu: float, shift: float, seed: int, replica: int, worker: int, seq: int) -> float:
-    """Compute time of task `seq` of `worker` in `replica`: shift + Exp(rate mu)."""
+    """Compute time of task `seq` of `worker` in `replica`: shift + Exp(rate mu), or for "pareto2"
+    a Pareto law of shape 2 (mu must be 2) and scale `shift`."""
     return float(lib().ora_delay(DELAYS[kind], float(mu), float(shift), int(seed), int(replica),
                                  int(worker), int(seq)))
 

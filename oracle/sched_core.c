@@ -14,6 +14,8 @@
  *   ora_delay              X = Delta + E/mu: per-minibatch compute time, i.i.d. over workers and
  *                          minibatches (Section 3.1, modelling assumptions; Exp(mu) has mean 1/mu,
  *                          Corollary 1; shifted exponential of Lemma 4)
+ *                          Pareto with shape 2 and scale x_m (the heavy-tailed law of the paper's
+ *                          runtime simulations, Figs. 4-5): X = x_m / sqrt(u), P(X > x) = (x_m/x)^2
  *   ora_minibatch_indices  m uniform draws with replacement from the n samples (Section 2)
  *   ora_schedule_*         Section 2.2: K-sync, K-batch-sync, K-async, K-batch-async, with K
  *                          possibly raised at wall-clock checkpoints (Algorithm 1's interval
@@ -27,7 +29,7 @@
 #define ORA_EXPORT __attribute__((visibility("default")))
 
 enum { ORA_KSYNC = 0, ORA_KBATCHSYNC = 1, ORA_KASYNC = 2, ORA_KBATCHASYNC = 3 };
-enum { ORA_DELAY_EXP = 0, ORA_DELAY_SHIFTED_EXP = 1 };
+enum { ORA_DELAY_EXP = 0, ORA_DELAY_SHIFTED_EXP = 1, ORA_DELAY_PARETO2 = 2 };
 
 /* ------------------------------------------------------------------------------------------
  * Philox4x32-10.  One round: the 32x32->64 products of counter words 0 and 2 with the two
@@ -93,10 +95,18 @@ ORA_EXPORT double ora_neg_log_uniform(uint32_t x0, uint32_t x1) {
     return fma((double)(53 - b), LN2, -lnf);
 }
 
+/* u = (2k+1) / 2^53 in (0,1), exact in fp64: the same uniform that ora_neg_log_uniform takes the log of */
+ORA_EXPORT double ora_uniform(uint32_t x0, uint32_t x1) {
+    uint64_t k = ((uint64_t)x0 << 20) | ((uint64_t)x1 >> 12);
+    return (double)(2u * k + 1u) * 0x1p-53;
+}
+
 ORA_EXPORT double ora_delay(int kind, double mu, double shift, uint64_t seed, uint32_t replica,
                             uint32_t worker, uint32_t seq) {
     uint32_t x[4];
     stream_words(seed, 0u, 0u, replica, worker, seq, x);
+    if (kind == ORA_DELAY_PARETO2)          /* shape 2 (given as mu), scale x_m (given as shift) */
+        return shift / sqrt(ora_uniform(x[0], x[1]));
     double e = ora_neg_log_uniform(x[0], x[1]);
     double base = (kind == ORA_DELAY_SHIFTED_EXP) ? shift : 0.0;
     return base + e / mu;

@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libstraggler_sim.so")
 
 VARIANTS = {"ksync": 0, "kbatchsync": 1, "kasync": 2, "kbatchasync": 3}
 MODELS = {"none": 0, "lsq": 1, "logistic": 2, "softmax": 3, "mlp2": 4}
-DELAYS = {"exp": 0, "shifted_exp": 1}
+DELAYS = {"exp": 0, "shifted_exp": 1, "pareto2": 2}
 STATUS = {0: "SIM_OK", 1: "SIM_ERR_ARG", 2: "SIM_ERR_ALLOC", 3: "SIM_ERR_CUDA", 4: "SIM_ERR_TIMEOUT",
           5: "SIM_ERR_STATE", 6: "SIM_ERR_INTERNAL"}
 

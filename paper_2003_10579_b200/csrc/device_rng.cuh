@@ -4,6 +4,8 @@
 // ((tag << 24) | chunk, task sequence number, worker, global replica id).  tag 0 / chunk 0 gives
 // the delay of a task, tag 1 / chunk c gives minibatch draws 4c .. 4c+3 of that task.
 //
+// A third law, Pareto with shape 2 (the heavy-tailed case of the paper's runtime simulations), is
+// X = x_m / sqrt(u) with the same u.
 // The delay X = shift + E / mu uses E = -ln(u) evaluated by a fixed sequence of integer
 // operations and round-to-nearest fp64 operations (explicit intrinsics, so that the compiler
 // neither contracts nor reorders them): the same inputs give the same bits on any IEEE machine,
@@ -64,13 +66,19 @@ __device__ __forceinline__ double neg_log_uniform(uint32_t x0, uint32_t x1) {
   return __fma_rn((double)(53 - b), __longlong_as_double(0x3FE62E42FEFA39EFll), -lnf);
 }
 
-struct DelayLaw { int shifted; double mu; double shift; };
+// kind: 0 = Exp(mu), 1 = shift + Exp(mu), 2 = Pareto of shape 2 and scale `shift`
+struct DelayLaw { int kind; double mu; double shift; };
 
 __device__ __forceinline__ double draw_delay(const DelayLaw& law, uint64_t seed, uint32_t replica,
                                              uint32_t worker, uint32_t seq) {
   const U4 x = stream_block(seed, 0u, 0u, replica, worker, seq);
+  if (law.kind == 2) {   // Pareto(2, x_m): X = x_m / sqrt(u), u = (2k+1)/2^53 exact; sqrt and divide are IEEE
+    const unsigned long long k = ((unsigned long long)x.x << 20) | ((unsigned long long)x.y >> 12);
+    const double u = __dmul_rn((double)(2ull * k + 1ull), 1.1102230246251565e-16 /* 2^-53 */);
+    return __ddiv_rn(law.shift, __dsqrt_rn(u));
+  }
   const double e = neg_log_uniform(x.x, x.y);
-  return __dadd_rn(law.shifted ? law.shift : 0.0, __ddiv_rn(e, law.mu));
+  return __dadd_rn(law.kind == 1 ? law.shift : 0.0, __ddiv_rn(e, law.mu));
 }
 
 // Draw q of the minibatch of task (replica, worker, seq): floor(u32 * n / 2^32), n <= 2^32.

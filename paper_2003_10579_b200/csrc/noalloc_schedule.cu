@@ -216,7 +216,10 @@ sim_status sim_schedule_noalloc(int32_t P, int32_t K, sim_variant variant, sim_d
   if (iters < 1 || iters > ((int64_t)1 << 31)) return na_fail(SIM_ERR_ARG, "iters must be in [1, 2^31]");
   if (replica_base < 0 || replica_base + (int64_t)n_replicas > (int64_t)1 << 32)
     return na_fail(SIM_ERR_ARG, "global replica ids must fit in 32 bits");
-  if (delay.kind != SIM_DELAY_EXP && delay.kind != SIM_DELAY_SHIFTED_EXP) return na_fail(SIM_ERR_ARG, "unknown delay kind");
+  if (delay.kind != SIM_DELAY_EXP && delay.kind != SIM_DELAY_SHIFTED_EXP && delay.kind != SIM_DELAY_PARETO2)
+    return na_fail(SIM_ERR_ARG, "unknown delay kind");
+  if (delay.kind == SIM_DELAY_PARETO2 && !(delay.mu == 2.0 && delay.shift > 0.0 && std::isfinite(delay.shift)))
+    return na_fail(SIM_ERR_ARG, "the Pareto law needs shape mu = 2 and a finite scale (shift) > 0");
   if (!(delay.mu > 0.0)) return na_fail(SIM_ERR_ARG, "delay rate mu must be > 0");
   if (delay.kind == SIM_DELAY_SHIFTED_EXP && !(delay.shift >= 0.0 && std::isfinite(delay.shift)))
     return na_fail(SIM_ERR_ARG, "delay shift must be finite and >= 0");
@@ -233,7 +236,7 @@ sim_status sim_schedule_noalloc(int32_t P, int32_t K, sim_variant variant, sim_d
 
   NaArgs a{};
   a.variant = (int)variant; a.P = P; a.K_fixed = K; a.K0 = growing ? K0 : 0; a.t_interval = growing ? t_interval : 0.0;
-  a.law.shifted = delay.kind == SIM_DELAY_SHIFTED_EXP; a.law.mu = delay.mu; a.law.shift = delay.shift;
+  a.law.kind = (int)delay.kind; a.law.mu = delay.mu; a.law.shift = delay.shift;
   a.seed = seed; a.R = n_replicas; a.replica_base = (uint32_t)replica_base; a.J = iters;
   a.K_stride = growing ? P : K; a.scratch = scratch;
   a.t = t; a.K_used = K_used; a.worker = worker; a.stale = stale; a.seq = seq;

@@ -105,7 +105,13 @@ long long model_params(const sim_problem& p) {
 }
 
 sim_status check_delay(const sim_handle* h, const sim_delay& dl) {
-  if (dl.kind != SIM_DELAY_EXP && dl.kind != SIM_DELAY_SHIFTED_EXP) return fail(h, SIM_ERR_ARG, "unknown delay kind");
+  if (dl.kind != SIM_DELAY_EXP && dl.kind != SIM_DELAY_SHIFTED_EXP && dl.kind != SIM_DELAY_PARETO2)
+    return fail(h, SIM_ERR_ARG, "unknown delay kind");
+  if (dl.kind == SIM_DELAY_PARETO2) {
+    if (dl.mu != 2.0) return fail(h, SIM_ERR_ARG, "the Pareto law is built for shape mu = 2 only");
+    if (!(dl.shift > 0.0 && std::isfinite(dl.shift))) return fail(h, SIM_ERR_ARG, "the Pareto scale (shift) must be finite and > 0");
+    return SIM_OK;
+  }
   if (!(dl.mu > 0.0)) return fail(h, SIM_ERR_ARG, "delay rate mu must be > 0");
   if (dl.kind == SIM_DELAY_SHIFTED_EXP && !(dl.shift >= 0.0 && std::isfinite(dl.shift)))
     return fail(h, SIM_ERR_ARG, "delay shift must be finite and >= 0");
@@ -358,7 +364,7 @@ sim_status sim_run(sim_handle* h, int64_t iters) {
 
   ScheduleArgs sa{};
   sa.variant = h->variant; sa.P = h->P; sa.K_fixed = h->K; sa.K0 = h->K0; sa.t_interval = h->t_interval;
-  sa.law.shifted = h->delay.kind == SIM_DELAY_SHIFTED_EXP; sa.law.mu = h->delay.mu; sa.law.shift = h->delay.shift;
+  sa.law.kind = (int)h->delay.kind; sa.law.mu = h->delay.mu; sa.law.shift = h->delay.shift;
   sa.seed = h->seed; sa.R = h->R; sa.replica_base = h->replica_base;
   sa.j0 = h->n_updates; sa.iters = iters; sa.cap = h->cap; sa.K_stride = h->K_stride; sa.n_slots = h->n_slots;
   sa.s = h->s; sa.tau = h->tau; sa.f = h->f; sa.wslot = h->wslot; sa.cur_slot = h->cur_slot;
@@ -473,7 +479,7 @@ sim_status sim_draw_delays(sim_delay delay, uint64_t seed, int64_t replica_base,
   if (st != SIM_OK) return st;
   if (!out || n_replicas < 1 || P < 1 || n_seq < 1 || replica_base < 0 || replica_base + (int64_t)n_replicas > (int64_t)1 << 32)
     return fail(nullptr, SIM_ERR_ARG, "sim_draw_delays: bad argument");
-  DelayLaw law{delay.kind == SIM_DELAY_SHIFTED_EXP, delay.mu, delay.shift};
+  DelayLaw law{(int)delay.kind, delay.mu, delay.shift};
   draw_delays_kernel<<<592, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(law, seed, (uint32_t)replica_base, n_replicas, P, n_seq, out);
   CUDA_TRY(nullptr, cudaGetLastError());
   return SIM_OK;

@@ -14,7 +14,7 @@ def B():
     return binding
 
 
-@pytest.mark.parametrize("kind,mu,shift", [("exp", 1.0, 0.0), ("shifted_exp", 2.0, 1.0), ("exp", 0.37, 0.0)])
+@pytest.mark.parametrize("kind,mu,shift", [("exp", 1.0, 0.0), ("shifted_exp", 2.0, 1.0), ("exp", 0.37, 0.0), ("pareto2", 2.0, 1.0), ("pareto2", 2.0, 0.3)])
 def test_delay_draws_bit_exact(B, kind, mu, shift):
     R, P, S, base, seed = 5, 7, 300, 3, 12345678901234
     got = B.draw_delays(kind, mu, shift, seed, base, R, P, S)
@@ -73,6 +73,11 @@ def test_schedule_ties(B, variant):
     check(B, variant, 5, 3, "shifted_exp", float("inf"), 0.5, R=2, J=12)
 
 
+@pytest.mark.parametrize("variant", list(core.VARIANTS))
+def test_schedule_under_pareto_delays(B, variant):
+    check(B, variant, 16, 5, "pareto2", 2.0, 1.0, seed=8, R=17, J=200, base=4)
+
+
 def test_first_workload_schedule_all_replicas(B):
     """K-sync, P=4, K=2, Exp(1), 64 replicas x 200 iterations, seed 0."""
     check(B, "ksync", 4, 2, R=64, J=200)
@@ -82,7 +87,8 @@ def test_bad_arguments_are_refused(B):
     S = B.Simulation
     base = dict(P=4, K=2, variant="ksync", delay_kind="exp", mu=1.0, eta=0.1, m=4, seed=0, n_replicas=2)
     for bad in (dict(P=0), dict(P=33), dict(K=0), dict(K=5), dict(m=0), dict(n_replicas=0), dict(mu=0.0),
-                dict(mu=float("nan")), dict(delay_kind="shifted_exp", shift=-1.0), dict(replica_base=2**32)):
+                dict(mu=float("nan")), dict(delay_kind="shifted_exp", shift=-1.0), dict(replica_base=2**32),
+                dict(delay_kind="pareto2", mu=3.0, shift=1.0), dict(delay_kind="pareto2", mu=2.0, shift=0.0)):
         with pytest.raises(B.SimError) as e:
             S(None, **{**base, **bad})
         assert e.value.status == 1

@@ -153,3 +153,15 @@ def test_minibatch_indices_formula_and_uniformity():
     assert chi2 < stats.chi2.ppf(0.9999, 63)
     # a prefix property: the first m' draws of a task do not depend on m
     assert core.minibatch_indices(9, 4, 2, 6, n, 8).tolist() == want[:8]
+
+
+def test_pareto_delay_law():
+    """Pareto(shape 2, scale x_m): P(X > x) = (x_m / x)^2, median x_m sqrt(2); X = x_m / sqrt(u)."""
+    xm = 1.5
+    x = np.array([core.delay("pareto2", 2.0, xm, 21, r, w, s) for r in range(30) for w in range(8) for s in range(400)])
+    assert x.min() >= xm
+    assert stats.kstest(x / xm, "pareto", args=(2.0,)).pvalue > 1e-4
+    assert abs(np.median(x) - xm * math.sqrt(2.0)) < 0.02 * xm
+    w = py_philox([21, 0], [0, 3, 2, 1])
+    k = (w[0] << 20) | (w[1] >> 12)
+    assert core.delay("pareto2", 2.0, xm, 21, 1, 2, 3) == xm / math.sqrt((2 * k + 1) / 2.0**53)

@@ -237,3 +237,18 @@ def test_bulk_schedule_equals_event_simulator(variant, P, K, K0, ti):
         ev = sim.trace_arrays(K_stride=tr["worker"].shape[2])
         for k in ("t", "K", "worker", "stale", "seq"):
             assert np.array_equal(tr[k][r], ev[k]), (variant, k)
+
+
+def test_ksync_order_statistics_under_pareto():
+    """Lemma 1 holds for any law: T = X_{K:P}.  Pareto(2,1): the minimum of P is Pareto(2P,1), the
+    maximum has CDF (1 - x^-2)^P (the heavy-tailed case of the paper's runtime simulations)."""
+    from scipy import stats
+    P = 8
+    Tmin = iteration_times(bulk("ksync", P, 1, "pareto2", 2.0, 1.0, seed=80, R=64, J=300)).ravel()
+    assert stats.kstest(Tmin, "pareto", args=(2.0 * P,)).pvalue > 1e-4
+    Tmax = iteration_times(bulk("ksync", P, P, "pareto2", 2.0, 1.0, seed=81, R=64, J=300)).ravel()
+    assert stats.kstest(Tmax, lambda x: (1.0 - np.minimum(1.0, x ** -2.0)) ** P).pvalue > 1e-4
+    # K-batch-async: long-run K E[X] / P with E[X] = 2 (Lemma 5; infinite variance, so a loose check)
+    tr = bulk("kbatchasync", 16, 4, "pareto2", 2.0, 1.0, seed=82, R=64, J=4000)
+    rate = (tr["t"][:, -1] - tr["t"][:, 499]) / 3500
+    assert abs(np.median(rate) - 4 * 2.0 / 16) < 0.05
