@@ -142,6 +142,15 @@ sim_status sim_get_trace(const sim_handle* h, double* t /*[R][J]*/, float* loss 
 /* Current parameters w_j of every replica into a DEVICE buffer [R][n_params]. */
 sim_status sim_get_params(const sim_handle* h, float* w);
 
+/*
+ * Full-data empirical risk F(w_j) = (1/N) sum_n f(w_j, xi_n) (Eq. 1) of every replica's current
+ * parameters into a DEVICE buffer [R]: the "error" of Section 2.3, for error-versus-wall-clock
+ * curves (call it between sim_run calls; the clock of the same update is in the trace).  One dense
+ * product over all replicas, fp32 logits, fp64 sums in a fixed order.  Built for LSQ, LOGISTIC and
+ * SOFTMAX (SIM_ERR_ARG otherwise).  Enqueued on the handle's stream; does not wait.
+ */
+sim_status sim_eval_loss(sim_handle* h, float* loss);
+
 /* Number of parameters of the handle's model (0 for SIM_NONE). */
 int64_t sim_n_params(const sim_handle* h);
 

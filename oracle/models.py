@@ -88,3 +88,13 @@ def loss_and_grad(model: str, w: np.ndarray, Xb: np.ndarray, yb: np.ndarray, n_c
                             (Hh.T @ D2).reshape(-1), D2.sum(axis=0)]) / m
         return float(loss.sum()), g
     raise ValueError(model)
+
+
+def full_loss(model: str, w: np.ndarray, X: np.ndarray, y: np.ndarray, n_classes: int = 1, hidden: int = 0,
+              bf16: bool = True, rows: int = 8192) -> float:
+    """Empirical risk F(w) = (1/N) sum_n f(w, xi_n) over the whole data set (Eq. 1), fp64, in row
+    blocks so that a large X needs no fp64 copy."""
+    total = 0.0
+    for a in range(0, X.shape[0], rows):
+        total += loss_and_grad(model, w, X[a:a + rows], y[a:a + rows], n_classes, hidden, bf16)[0]
+    return total / X.shape[0]

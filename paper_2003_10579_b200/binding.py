@@ -20,7 +20,7 @@ STATUS = {0: "SIM_OK", 1: "SIM_ERR_ARG", 2: "SIM_ERR_ALLOC", 3: "SIM_ERR_CUDA", 
           5: "SIM_ERR_STATE", 6: "SIM_ERR_INTERNAL"}
 
 EXPORTS = ["sim_create", "sim_set_params", "sim_set_adasync", "sim_set_tuning", "sim_reserve", "sim_run",
-           "sim_trace_size", "sim_get_trace", "sim_get_params", "sim_n_params", "sim_last_error",
+           "sim_trace_size", "sim_get_trace", "sim_get_params", "sim_eval_loss", "sim_n_params", "sim_last_error",
            "sim_destroy", "sim_draw_delays", "sim_draw_indices", "sim_simulate_host", "sim_sweep_host", "sim_schedule_noalloc",
            "sim_noalloc_last_error"]
 
@@ -57,6 +57,7 @@ def _load():
     L.sim_trace_size.argtypes = [vp, C.POINTER(i64), C.POINTER(i32)]
     L.sim_get_trace.argtypes = [vp] * 8
     L.sim_get_params.argtypes = [vp, vp]
+    L.sim_eval_loss.argtypes = [vp, vp]
     L.sim_n_params.argtypes = [vp]
     L.sim_n_params.restype = i64
     L.sim_last_error.argtypes = [vp]
@@ -176,6 +177,16 @@ class Simulation:
         w = torch.empty((self.R, self.n_params), dtype=torch.float32, device=self.device)
         _check(lib.sim_get_params(self._h, _ptr(w)), self._h)
         return w.cpu().numpy() if to_numpy else w
+
+    def eval_loss(self, to_numpy=True):
+        """Full-data risk F(w_j) of every replica's current parameters."""
+        out = torch.empty((self.R,), dtype=torch.float32, device=self.device)
+        _check(lib.sim_eval_loss(self._h, _ptr(out)), self._h)
+        if self.stream is not None:
+            self.stream.synchronize()
+        else:
+            torch.cuda.synchronize()
+        return out.cpu().numpy() if to_numpy else out
 
     def close(self):
         if self._h:

@@ -12,6 +12,7 @@
 #include "linear_kernel.cuh"
 #include "softmax_kernel.cuh"
 #include "mlp_tc_kernel.cuh"
+#include "eval_kernel.cuh"
 
 using namespace ssim;
 
@@ -65,6 +66,7 @@ struct sim_handle {
   MlpScratch mlp{};
   MlpMaps mlp_maps{};
   int* err = nullptr;
+  double* eval_partial = nullptr;   // [row blocks][R], made on the first sim_eval_loss
   TraceBuffers tr;
   bool poisoned = false;
   mutable std::string last_error;
@@ -223,6 +225,7 @@ void free_all(sim_handle* h) {
   cudaFree(h->s); cudaFree(h->tau); cudaFree(h->f); cudaFree(h->wslot); cudaFree(h->cur_slot);
   cudaFree(h->begin_slot); cudaFree(h->clock); cudaFree(h->w_state); cudaFree(h->pool); cudaFree(h->err);
   mlp_scratch_free(h->mlp);
+  cudaFree(h->eval_partial);
   cudaFree(h->tr.t); cudaFree(h->tr.loss); cudaFree(h->tr.dist2); cudaFree(h->tr.K_used);
   cudaFree(h->tr.worker); cudaFree(h->tr.stale); cudaFree(h->tr.seq); cudaFree(h->tr.snap_slot);
   cudaFree(h->tr.new_slot);
@@ -459,6 +462,32 @@ sim_status sim_get_params(const sim_handle* h, float* w) {
     CUDA_TRY(h, cudaMemcpyAsync(w, h->w_state, (size_t)h->R * h->n_params * sizeof(float), cudaMemcpyDeviceToDevice, h->stream));
   }
   CUDA_TRY(h, cudaStreamSynchronize(h->stream));
+  return SIM_OK;
+}
+
+sim_status sim_eval_loss(sim_handle* h, float* loss) {
+  if (!h) return fail(nullptr, SIM_ERR_ARG, "handle is NULL");
+  if (!loss) return fail(h, SIM_ERR_ARG, "loss is NULL");
+  if (h->poisoned) return fail(h, SIM_ERR_STATE, "the handle failed earlier");
+  const sim_model mdl = h->prob.model;
+  if (mdl != SIM_LSQ && mdl != SIM_LOGISTIC && mdl != SIM_SOFTMAX)
+    return fail(h, SIM_ERR_ARG, "sim_eval_loss is built for the linear models (LSQ, logistic, softmax)");
+  EvalArgs e{};
+  e.X = h->prob.X;
+  e.y = mdl == SIM_LSQ ? static_cast<const void*>(h->prob.y) : static_cast<const void*>(h->prob.label);
+  e.n = h->prob.n; e.d = h->prob.d; e.C = mdl == SIM_SOFTMAX ? h->prob.n_classes : 1; e.model = (int)mdl; e.R = h->R;
+  e.RB = EV_BN / e.C;
+  e.w_state = h->uses_pool ? nullptr : h->w_state;
+  e.pool = h->uses_pool ? h->pool : nullptr;
+  e.cur_slot = h->cur_slot; e.n_slots = h->n_slots; e.n_params = h->n_params; e.slot_stride = h->slot_stride;
+  e.row_blocks = (int)((h->prob.n + EV_BM - 1) / EV_BM);
+  if (!h->eval_partial) CUDA_TRY(h, dev_alloc(&h->eval_partial, (size_t)e.row_blocks * h->R, h->stream, false));
+  e.partial = h->eval_partial; e.out = loss;
+  dim3 grid((unsigned)e.row_blocks, (unsigned)((h->R + e.RB - 1) / e.RB));
+  eval_loss_kernel<<<grid, 256, 0, h->stream>>>(e);
+  CUDA_TRY(h, cudaGetLastError());
+  eval_loss_finish_kernel<<<(h->R + 127) / 128, 128, 0, h->stream>>>(e);
+  CUDA_TRY(h, cudaGetLastError());
   return SIM_OK;
 }
 

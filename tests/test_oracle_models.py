@@ -201,3 +201,20 @@ def test_error_floor_scales_as_one_over_K():
 
     ratio = floor(2) / floor(4)
     assert 1.4 < ratio < 2.8
+
+
+def test_full_loss_is_the_mean_of_the_per_sample_losses_and_blocks_do_not_matter():
+    """Eq. 1: F(w) = (1/N) sum_n f(w, xi_n)."""
+    data = inputs.make_lsq(1000, 16, 0.3, 11)
+    w = np.linspace(-1, 1, 16).astype(np.float32)
+    r = data["X"].astype(np.float64) @ w.astype(np.float64) - data["y"]
+    want = float(np.mean(0.5 * r * r))
+    assert abs(models.full_loss("lsq", w, data["X"], data["y"]) - want) < 1e-14 * want
+    assert abs(models.full_loss("lsq", w, data["X"], data["y"], rows=77) - want) < 1e-13 * want
+    mix = inputs.make_mixture(500, 16, 4, 0.5, 12)
+    W = (0.1 * np.arange(64) % 0.7).astype(np.float32)
+    per = [models.loss_and_grad("softmax", W, mix["X"][i:i + 1], mix["y"][i:i + 1], 4)[0] for i in range(500)]
+    assert abs(models.full_loss("softmax", W, mix["X"], mix["y"], 4, rows=64) - np.mean(per)) < 1e-13
+    # at the least-squares solution of noiseless data the risk vanishes
+    clean = inputs.make_lsq(400, 8, 0.0, 13)
+    assert models.full_loss("lsq", clean["w_star"], clean["X"], clean["y"]) < 1e-12
