@@ -20,7 +20,13 @@ Readings taken where the text leaves a choice:
     update reads w_{j+1};
   * a cancelled task still consumes its sequence number;
   * with a K schedule, K for an update is K0 doubled once per whole interval elapsed at the
-    previous update's time, capped at P (Algorithm 1's interval structure).
+    previous update's time, capped at P (Algorithm 1's interval structure);
+  * with k_rule="loss" (Algorithm 1 and Section 6 as printed): whenever an update starts in a later
+    interval than the one K was last set in, and K < P, K is recomputed from the full-data risk
+    F(w_start) of the parameters at that moment (F* taken as 0, F rounded to fp32 as a device
+    computes it): K = K0 sqrt(F(w_0)/F(w_start)) for K-batch-sync, K-async, K-batch-async; for K-sync
+    the root of K^2/(P-K) = K0^2/(P-K0) F(w_0)/F(w_start).  The real value is rounded half up and
+    K never decreases nor exceeds P.
 """
 from __future__ import annotations
 
@@ -31,9 +37,27 @@ import numpy as np
 from . import core, models
 
 
+def adasync_next_K(variant, K0, P, K_prev, F0, F):
+    """The rule of Section 6 / Algorithm 1 for one interval boundary (fp64 on fp32 risks)."""
+    F0, F = float(np.float32(F0)), float(np.float32(F))
+    if not (F > 0.0 and math.isfinite(F) and math.isfinite(F0)):
+        return P
+    ratio = F0 / F
+    if variant == "ksync":
+        if K0 >= P:
+            return P
+        c = (float(K0 * K0) / float(P - K0)) * ratio        # K^2 = c (P - K)
+        disc = c * c + (4.0 * c) * float(P)
+        k_real = (math.sqrt(disc) + (-c)) * 0.5
+    else:
+        k_real = float(K0) * math.sqrt(ratio)
+    K = int(math.floor(k_real + 0.5)) if k_real < 1e9 else P
+    return min(P, max(K_prev, K))
+
+
 class OracleReplica:
     def __init__(self, *, model, X, y, w0, P, K, variant, delay_kind, mu, shift=0.0, eta, m, seed,
-                 replica, n_classes=1, hidden=0, w_ref=None, K0=0, t_interval=0.0, bf16=True):
+                 replica, n_classes=1, hidden=0, w_ref=None, K0=0, t_interval=0.0, bf16=True, k_rule="doubling"):
         assert variant in core.VARIANTS and 1 <= P and 1 <= m
         self.model, self.X, self.y = model, X, y
         self.n = 0 if X is None else X.shape[0]
@@ -43,6 +67,8 @@ class OracleReplica:
         self.eta = float(np.float32(eta))
         self.m, self.seed, self.r = m, seed, replica
         self.K0, self.t_interval = K0, t_interval
+        self.k_rule, self.K_cur, self.q_last, self.F0 = k_rule, K0, 0, None
+        self.k_events = []               # (update index, F(w_start), new K) at every recomputation
         self.w_ref = None if w_ref is None else np.asarray(w_ref, np.float64)
         self.w = None if w0 is None else np.array(w0, dtype=np.float32)   # w_j
         self.j = 0
@@ -64,6 +90,16 @@ class OracleReplica:
     def _K_now(self):
         if not self.t_interval > 0.0:
             return self.K_fixed
+        if self.k_rule == "loss":
+            if self.F0 is None:
+                self.F0 = np.float32(self._risk())
+            q = math.floor(self.t / self.t_interval)
+            if q > self.q_last and self.K_cur < self.P:
+                F = np.float32(self._risk())
+                self.K_cur = adasync_next_K(self.variant, self.K0, self.P, self.K_cur, self.F0, F)
+                self.q_last = q
+                self.k_events.append((self.j, float(F), self.K_cur))
+            return self.K_cur
         q = math.floor(self.t / self.t_interval)
         K = self.K0
         while q > 0 and K < self.P:
@@ -71,6 +107,9 @@ class OracleReplica:
         return min(K, self.P)
 
     # -- numerics -------------------------------------------------------------------------
+    def _risk(self):
+        return models.full_loss(self.model, self.w, self.X, self.y, self.n_classes, self.hidden, self.bf16)
+
     def _gradient(self, w_at, i, seq):
         idx = core.minibatch_indices(self.seed, self.r, i, seq, self.n, self.m)
         return models.loss_and_grad(self.model, w_at, self.X[idx], self.y[idx], self.n_classes,

@@ -1,4 +1,6 @@
 """Pins for the oracle's gradients and for the update rule of Eq. 2 / Eq. 3.  CPU only."""
+import math
+
 import numpy as np
 import pytest
 import torch
@@ -218,3 +220,53 @@ def test_full_loss_is_the_mean_of_the_per_sample_losses_and_blocks_do_not_matter
     # at the least-squares solution of noiseless data the risk vanishes
     clean = inputs.make_lsq(400, 8, 0.0, 13)
     assert models.full_loss("lsq", clean["w_star"], clean["X"], clean["y"]) < 1e-12
+
+
+def test_adasync_rule_closed_forms():
+    """Section 6: K = K0 sqrt(F0/F) (three variants); K-sync: K^2/(P-K) = K0^2/(P-K0) F0/F."""
+    from oracle.sim import adasync_next_K
+    import math
+    for v in ("kbatchsync", "kasync", "kbatchasync"):
+        assert adasync_next_K(v, 1, 16, 1, 4.0, 1.0) == 2          # ratio 4 doubles K
+        assert adasync_next_K(v, 2, 16, 2, 9.0, 1.0) == 6
+        assert adasync_next_K(v, 1, 8, 1, 1.0, 1.0) == 1            # no progress, no change
+        assert adasync_next_K(v, 1, 8, 3, 1.0, 1.0) == 3            # never decreases
+        assert adasync_next_K(v, 1, 8, 1, 1.0, 1e-6) == 8           # capped at P
+        assert adasync_next_K(v, 1, 8, 1, 1.0, 0.0) == 8            # F = F* = 0: fully synchronous
+    rng = np.random.default_rng(5)
+    for _ in range(200):
+        P = int(rng.integers(2, 33)); K0 = int(rng.integers(1, P)); ratio = float(np.float32(10 ** rng.uniform(0, 3)))
+        c = K0 * K0 / (P - K0) * ratio
+        k_real = (math.sqrt(c * c + 4 * c * P) - c) / 2               # root of K^2 + cK - cP
+        assert abs(k_real ** 2 / (P - k_real) - c) < 1e-9 * c and K0 - 1e-9 <= k_real < P
+        got = adasync_next_K("ksync", K0, P, K0, ratio, 1.0)
+        if abs(k_real + 0.5 - round(k_real + 0.5)) > 1e-6:
+            assert got == min(P, max(K0, math.floor(k_real + 0.5)))
+    assert adasync_next_K("ksync", 4, 4, 4, 5.0, 1.0) == 4
+    assert adasync_next_K("ksync", 1, 8, 1, 1.0, 1.0) == 1
+
+
+@pytest.mark.parametrize("variant", list(core.VARIANTS))
+def test_loss_driven_adasync_in_the_simulator(variant):
+    data = inputs.make_lsq(512, 16, 0.05, 14)
+    kw = dict(model="lsq", X=data["X"], y=data["y"], w0=np.zeros(16, np.float32), P=8, K=1, variant=variant,
+              delay_kind="shifted_exp", mu=2.0, shift=0.5, eta=0.05, m=4, seed=6, replica=3)
+    sim = OracleReplica(K0=1, t_interval=4.0, k_rule="loss", **kw).run(250)
+    tr = sim.trace_arrays()
+    K = tr["K"].astype(int)
+    assert K[0] == 1 and np.all(np.diff(K) >= 0) and K.max() <= 8 and K.max() > 1
+    # K changes only at an update that starts in a new interval, and to the rule's value
+    t_start = np.concatenate([[0.0], tr["t"][:-1]])
+    for j in np.nonzero(np.diff(K))[0] + 1:
+        assert math.floor(t_start[j] / 4.0) > math.floor(t_start[j - 1] / 4.0)
+    from oracle.sim import adasync_next_K
+    F0 = np.float32(models.full_loss("lsq", np.zeros(16, np.float32), data["X"], data["y"]))
+    k_prev = 1
+    for (j, F, k_new) in sim.k_events:
+        assert k_new == adasync_next_K(variant, 1, 8, k_prev, F0, F) and K[j] == k_new
+        k_prev = k_new
+    # an interval that never ends leaves K at K0: the fixed-K run, bit for bit
+    a = OracleReplica(K0=2, t_interval=1e300, k_rule="loss", **{**kw, "K": 0}).run(60).trace_arrays(K_stride=8)
+    b = OracleReplica(**{**kw, "K": 2}).run(60).trace_arrays(K_stride=8)
+    for k in ("t", "K", "worker", "stale", "seq", "loss"):
+        assert np.array_equal(a[k], b[k]), k
