@@ -106,6 +106,18 @@ sim_status sim_set_params(sim_handle* h, const float* w0);
  * switches it off (fixed K from sim_create).  Only before the first sim_run. */
 sim_status sim_set_adasync(sim_handle* h, int32_t K0, double t_interval);
 
+/*
+ * AdaSync as printed (Algorithm 1; derivation in Section 6 and its appendix): start at K0; whenever
+ * an update starts in a later interval of length t_interval than the one K was last set in, and
+ * K < P, set K from the full-data risk F (Eq. 1, F* taken as 0) of the parameters at that moment:
+ *   K-batch-sync, K-async, K-batch-async:  K = K0 sqrt(F(w_0) / F(w_start))
+ *   K-sync:  the positive root of  K^2 / (P - K) = K0^2 / (P - K0) * F(w_0) / F(w_start)
+ * rounded half up, never decreasing, at most P.  Replicas pause at different updates, so sim_run
+ * proceeds in rounds (one per interval crossing) and synchronises the stream between rounds.  LSQ,
+ * LOGISTIC and SOFTMAX only (the rule needs sim_eval_loss).  Only before the first sim_run.
+ */
+sim_status sim_set_adasync_loss(sim_handle* h, int32_t K0, double t_interval);
+
 /* Optional performance knobs of the linear-model kernels (0 = chosen from d): depth of the
  * shared-memory ring that stages sample rows ahead of the arithmetic (2..8), rows per tile (2 or
  * 4) and threads per replica (256 or 512) where the kernel for that d offers the choice.

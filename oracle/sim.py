@@ -37,20 +37,24 @@ import numpy as np
 from . import core, models
 
 
-def adasync_next_K(variant, K0, P, K_prev, F0, F):
-    """The rule of Section 6 / Algorithm 1 for one interval boundary (fp64 on fp32 risks)."""
+def adasync_k_real(variant, K0, P, F0, F):
+    """The real-valued K of Section 6 / Algorithm 1 (fp64 on fp32 risks); inf once F reaches F* = 0."""
     F0, F = float(np.float32(F0)), float(np.float32(F))
     if not (F > 0.0 and math.isfinite(F) and math.isfinite(F0)):
-        return P
+        return math.inf
     ratio = F0 / F
     if variant == "ksync":
         if K0 >= P:
-            return P
+            return float(P)
         c = (float(K0 * K0) / float(P - K0)) * ratio        # K^2 = c (P - K)
         disc = c * c + (4.0 * c) * float(P)
-        k_real = (math.sqrt(disc) + (-c)) * 0.5
-    else:
-        k_real = float(K0) * math.sqrt(ratio)
+        return (math.sqrt(disc) + (-c)) * 0.5
+    return float(K0) * math.sqrt(ratio)
+
+
+def adasync_next_K(variant, K0, P, K_prev, F0, F):
+    """One interval boundary: the real value rounded half up, never decreasing, at most P."""
+    k_real = adasync_k_real(variant, K0, P, F0, F)
     K = int(math.floor(k_real + 0.5)) if k_real < 1e9 else P
     return min(P, max(K_prev, K))
 

@@ -19,7 +19,7 @@ DELAYS = {"exp": 0, "shifted_exp": 1, "pareto2": 2}
 STATUS = {0: "SIM_OK", 1: "SIM_ERR_ARG", 2: "SIM_ERR_ALLOC", 3: "SIM_ERR_CUDA", 4: "SIM_ERR_TIMEOUT",
           5: "SIM_ERR_STATE", 6: "SIM_ERR_INTERNAL"}
 
-EXPORTS = ["sim_create", "sim_set_params", "sim_set_adasync", "sim_set_tuning", "sim_reserve", "sim_run",
+EXPORTS = ["sim_create", "sim_set_params", "sim_set_adasync", "sim_set_adasync_loss", "sim_set_tuning", "sim_reserve", "sim_run",
            "sim_trace_size", "sim_get_trace", "sim_get_params", "sim_eval_loss", "sim_n_params", "sim_last_error",
            "sim_destroy", "sim_draw_delays", "sim_draw_indices", "sim_simulate_host", "sim_sweep_host", "sim_schedule_noalloc",
            "sim_noalloc_last_error"]
@@ -51,6 +51,7 @@ def _load():
                              i64, vp, C.POINTER(vp)]
     L.sim_set_params.argtypes = [vp, vp]
     L.sim_set_adasync.argtypes = [vp, i32, dbl]
+    L.sim_set_adasync_loss.argtypes = [vp, i32, dbl]
     L.sim_set_tuning.argtypes = [vp, i32, i32, i32]
     L.sim_reserve.argtypes = [vp, i64]
     L.sim_run.argtypes = [vp, i64]
@@ -140,6 +141,10 @@ class Simulation:
 
     def set_adasync(self, K0, t_interval):
         _check(lib.sim_set_adasync(self._h, K0, t_interval), self._h)
+
+    def set_adasync_loss(self, K0, t_interval):
+        """Algorithm 1 as printed: K follows the full-data risk at interval boundaries."""
+        _check(lib.sim_set_adasync_loss(self._h, K0, t_interval), self._h)
 
     def set_tuning(self, stages=0, tile_rows=0, threads=0):
         _check(lib.sim_set_tuning(self._h, stages, tile_rows, threads), self._h)

@@ -30,6 +30,8 @@ struct NumericArgs {
   uint32_t replica_base;
   int R;
   long long j0, iters, cap;
+  const long long* run_j0;   // optional per-replica [R] first update / update count of this launch (loss-driven K:
+  const long long* run_iters; // replicas pause at different updates); null: j0 / iters for all
   int K_stride;
   int is_async;
   int n_slots;
@@ -128,10 +130,10 @@ struct ScheduleWalk {
     if (nl >= (int)cur.K) { nl = 0; nj = j + 1; }
     if (nj < j_end) nxt = load(a, nj, nl);
   }
-  __device__ __forceinline__ void start(const NumericArgs& a, int r) {
-    row0 = (long long)r * a.cap; j = a.j0; j_end = a.j0 + a.iters; l = 0; k = 0;
+  __device__ __forceinline__ void start(const NumericArgs& a, int r, long long first, long long count) {
+    row0 = (long long)r * a.cap; j = first; j_end = first + count; l = 0; k = 0;
     tiles_per_task = (a.m + 0) ;   // set by caller (depends on T)
-    done = a.iters <= 0;
+    done = count <= 0;
     if (!done) { cur = load(a, j, 0); prefetch_next(a); }
   }
   __device__ __forceinline__ void advance(const NumericArgs& a) {
@@ -153,6 +155,7 @@ __global__ void __launch_bounds__(NT) linear1_kernel(NumericArgs a) {
   const int d = a.d, d4 = d >> 2, S = a.stages, m = a.m;
   const uint32_t rid = a.replica_base + (uint32_t)r;
   const uint32_t row_bytes = (uint32_t)d * 4u;
+  const long long my_j0 = a.run_j0 ? a.run_j0[r] : a.j0, my_iters = a.run_iters ? a.run_iters[r] : a.iters;
 
   extern __shared__ __align__(128) unsigned char smem[];
   // layout: [S] barriers | [S] TileInfo | y_stage [S][T] | red [2][NW][T] | misc [NW] | rows [S][T][d]
@@ -222,15 +225,15 @@ __global__ void __launch_bounds__(NT) linear1_kernel(NumericArgs a) {
     walk.advance(a);
   };
   if (warp == 0) {
-    walk.start(a, r);
+    walk.start(a, r, my_j0, my_iters);
     walk.tiles_per_task = (m + T - 1) / T;
     for (int s = 0; s < S - 1; ++s) issue_tile(s);
   }
   __syncthreads();
-  if (a.iters <= 0) return;
+  if (my_iters <= 0) return;
 
   float loss_acc = 0.f;
-  long long j = a.j0;
+  long long j = my_j0;
   bool failed = false;
   for (long long it = 0;; ++it) {
     const int st = (int)(it % S);

@@ -43,6 +43,16 @@ struct ScheduleArgs {
   uint8_t* snap_slot;        // [R][cap][K_stride] (asynchronous variants, else null)
   uint8_t* new_slot;         // [R][cap]
   int* err;
+  // loss-driven K (Algorithm 1): a replica's K changes only when an update starts in a later interval
+  // than the one K was last set in; the arrival process then pauses there until the risk is known
+  int adaptive;
+  long long target;          // every replica is advanced to this many updates in total
+  long long* done;           // [R] updates scheduled so far
+  long long* run_j0;         // [R] out: first update and number of updates scheduled by this launch
+  long long* run_iters;
+  int* K_cur;                // [R] K in force
+  long long* q_last;         // [R] interval index K was last set in
+  int* want_eval;            // [R] out: 1 if the replica paused because it needs a new K
 };
 
 // K in force for an update that starts at simulated time t (doubling once per elapsed interval).
@@ -101,15 +111,29 @@ __global__ void __launch_bounds__(128) schedule_kernel(ScheduleArgs a) {
   int cur = async ? a.cur_slot[r] : 0;
   double clock = a.clock[r];
 
-  if (async && a.j0 == 0) {   // every worker fetches w_0 and starts its first minibatch at t = 0
+  long long j = a.adaptive ? a.done[r] : a.j0;
+  const long long j_begin = j, j_end = a.adaptive ? a.target : a.j0 + a.iters;
+  int K_now = a.adaptive ? a.K_cur[r] : 0, want = 0;
+  long long q_last = a.adaptive ? a.q_last[r] : 0;
+  if (async && j == 0 && __all_sync(0xFFFFFFFFu, s == 0u)) {   // every worker fetches w_0 and starts its first minibatch at t = 0
     if (active) { f = __dadd_rn(0.0, draw_delay(a.law, a.seed, rid, lane, s)); s += 1; tau = 0; slot = 0; }
     cur = 0;
   }
   if (async && lane == 0) a.begin_slot[r] = (uint8_t)cur;
 
-  for (long long u = 0; u < a.iters; ++u) {
-    const long long j = a.j0 + u;
-    const int K = k_for_time(a, clock);
+  for (; j < j_end; ++j) {
+    int K;
+    if (a.adaptive) {
+      const double qd = floor(__ddiv_rn(clock, a.t_interval));
+      const long long q = qd > 9.0e18 ? 0x7FFFFFFFFFFFFFFFll : (long long)qd;
+      if (q > q_last) {
+        if (K_now < P) { want = 1; break; }     // the risk of w_j decides the next K
+        q_last = q;
+      }
+      K = K_now;
+    } else {
+      K = k_for_time(a, clock);
+    }
     const long long row = (long long)r * a.cap + j;
     uint16_t* wk = a.worker + row * a.K_stride;
     uint32_t* sl = a.stale + row * a.K_stride;
@@ -190,7 +214,52 @@ __global__ void __launch_bounds__(128) schedule_kernel(ScheduleArgs a) {
     a.tau[r * P + lane] = tau;
     if (async) { a.f[r * P + lane] = f; a.wslot[r * P + lane] = (uint8_t)slot; }
   }
-  if (lane == 0) { a.clock[r] = clock; if (async) a.cur_slot[r] = (uint8_t)cur; }
+  if (lane == 0) {
+    a.clock[r] = clock;
+    if (async) a.cur_slot[r] = (uint8_t)cur;
+    if (a.adaptive) {
+      a.run_j0[r] = j_begin; a.run_iters[r] = j - j_begin; a.done[r] = j;
+      a.q_last[r] = q_last; a.want_eval[r] = want;
+    }
+  }
+}
+
+// After the risk of the paused replicas is known: the rule of Section 6 / Algorithm 1.
+//   K-batch-sync, K-async, K-batch-async:  K = K0 sqrt(F(w_0) / F(w_start))
+//   K-sync:  K^2 / (P - K) = K0^2 / (P - K0) * F(w_0) / F(w_start)   (positive root)
+// rounded half up, never decreasing, at most P; F <= 0 (F* reached) gives P.  fp64 with explicit
+// round-to-nearest operations on the fp32 risks, so that the integer is reproducible elsewhere.
+__global__ void adasync_update_kernel(int variant, int P, int K0, double t_interval, int R, long long target,
+                                      const float* F0, const float* F, const double* clock, const long long* done,
+                                      int* K_cur, long long* q_last, int* want_eval, int* remaining) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= R) return;
+  if (want_eval[r]) {
+    const double f0 = (double)F0[r], f = (double)F[r];
+    int K = P;
+    if (f > 0.0 && isfinite(f) && isfinite(f0)) {
+      const double ratio = __ddiv_rn(f0, f);
+      double k_real;
+      if (variant == V_KSYNC) {
+        if (K0 >= P) k_real = (double)P;
+        else {
+          const double c = __dmul_rn(__ddiv_rn((double)(K0 * K0), (double)(P - K0)), ratio);
+          const double disc = __dadd_rn(__dmul_rn(c, c), __dmul_rn(__dmul_rn(4.0, c), (double)P));
+          k_real = __dmul_rn(__dadd_rn(__dsqrt_rn(disc), -c), 0.5);
+        }
+      } else {
+        k_real = __dmul_rn((double)K0, __dsqrt_rn(ratio));
+      }
+      K = k_real < 1e9 ? (int)floor(__dadd_rn(k_real, 0.5)) : P;
+    }
+    const int prev = K_cur[r];
+    K = K < prev ? prev : K;
+    K_cur[r] = K > P ? P : K;
+    const double qd = floor(__ddiv_rn(clock[r], t_interval));
+    q_last[r] = qd > 9.0e18 ? 0x7FFFFFFFFFFFFFFFll : (long long)qd;
+    want_eval[r] = 0;
+  }
+  if (done[r] < target) atomicAdd(remaining, 1);
 }
 
 // The raw draws, for checking the stream against another implementation.

@@ -67,6 +67,11 @@ struct sim_handle {
   MlpMaps mlp_maps{};
   int* err = nullptr;
   double* eval_partial = nullptr;   // [row blocks][R], made on the first sim_eval_loss
+  // loss-driven K (Algorithm 1): per-replica progress and K, risks at w_0 and at the last pause
+  bool ada_loss = false, F0_ready = false;
+  float* F0 = nullptr; float* Fcur = nullptr;
+  long long* done = nullptr; long long* run_j0 = nullptr; long long* run_iters = nullptr; long long* q_last = nullptr;
+  int* K_cur = nullptr; int* want_eval = nullptr; int* remaining = nullptr;
   TraceBuffers tr;
   bool poisoned = false;
   mutable std::string last_error;
@@ -225,10 +230,39 @@ void free_all(sim_handle* h) {
   cudaFree(h->s); cudaFree(h->tau); cudaFree(h->f); cudaFree(h->wslot); cudaFree(h->cur_slot);
   cudaFree(h->begin_slot); cudaFree(h->clock); cudaFree(h->w_state); cudaFree(h->pool); cudaFree(h->err);
   mlp_scratch_free(h->mlp);
-  cudaFree(h->eval_partial);
+  cudaFree(h->eval_partial); cudaFree(h->F0); cudaFree(h->Fcur); cudaFree(h->done); cudaFree(h->run_j0);
+  cudaFree(h->run_iters); cudaFree(h->q_last); cudaFree(h->K_cur); cudaFree(h->want_eval); cudaFree(h->remaining);
   cudaFree(h->tr.t); cudaFree(h->tr.loss); cudaFree(h->tr.dist2); cudaFree(h->tr.K_used);
   cudaFree(h->tr.worker); cudaFree(h->tr.stale); cudaFree(h->tr.seq); cudaFree(h->tr.snap_slot);
   cudaFree(h->tr.new_slot);
+}
+
+sim_status eval_into(sim_handle* h, float* loss) {
+  const sim_model mdl = h->prob.model;
+  if (mdl != SIM_LSQ && mdl != SIM_LOGISTIC && mdl != SIM_SOFTMAX)
+    return fail(h, SIM_ERR_ARG, "the full-data risk is built for the linear models (LSQ, logistic, softmax)");
+  EvalArgs e{};
+  e.X = h->prob.X;
+  e.y = mdl == SIM_LSQ ? static_cast<const void*>(h->prob.y) : static_cast<const void*>(h->prob.label);
+  e.n = h->prob.n; e.d = h->prob.d; e.C = mdl == SIM_SOFTMAX ? h->prob.n_classes : 1; e.model = (int)mdl; e.R = h->R;
+  e.RB = EV_BN / e.C;
+  e.w_state = h->uses_pool ? nullptr : h->w_state;
+  e.pool = h->uses_pool ? h->pool : nullptr;
+  e.cur_slot = h->cur_slot; e.n_slots = h->n_slots; e.n_params = h->n_params; e.slot_stride = h->slot_stride;
+  e.row_blocks = (int)((h->prob.n + EV_BM - 1) / EV_BM);
+  if (!h->eval_partial) CUDA_TRY(h, dev_alloc(&h->eval_partial, (size_t)e.row_blocks * h->R, h->stream, false));
+  e.partial = h->eval_partial; e.out = loss;
+  dim3 grid((unsigned)e.row_blocks, (unsigned)((h->R + e.RB - 1) / e.RB));
+  eval_loss_kernel<<<grid, 256, 0, h->stream>>>(e);
+  CUDA_TRY(h, cudaGetLastError());
+  eval_loss_finish_kernel<<<(h->R + 127) / 128, 128, 0, h->stream>>>(e);
+  CUDA_TRY(h, cudaGetLastError());
+  return SIM_OK;
+}
+
+__global__ void fill_int_kernel(int* p, int v, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) p[i] = v;
 }
 
 }  // namespace
@@ -334,7 +368,7 @@ sim_status sim_set_adasync(sim_handle* h, int32_t K0, double t_interval) {
   if (h->n_updates > 0 || h->cap > 0) return fail(h, SIM_ERR_STATE, "sim_set_adasync is only allowed before sim_reserve / sim_run");
   if (t_interval > 0.0) {
     if (K0 < 1 || K0 > h->P) return fail(h, SIM_ERR_ARG, "K0 must be in [1, P]");
-    h->K0 = K0; h->t_interval = t_interval; h->K_stride = h->P;
+    h->K0 = K0; h->t_interval = t_interval; h->K_stride = h->P; h->ada_loss = false;
   } else {
     h->K0 = 0; h->t_interval = 0.0; h->K_stride = h->K;
   }
@@ -374,11 +408,22 @@ sim_status sim_run(sim_handle* h, int64_t iters) {
   sa.begin_slot = h->begin_slot; sa.clock = h->clock;
   sa.t = h->tr.t; sa.K_used = h->tr.K_used; sa.worker = h->tr.worker; sa.stale = h->tr.stale; sa.seq = h->tr.seq;
   sa.snap_slot = h->tr.snap_slot; sa.new_slot = h->tr.new_slot; sa.err = h->err;
+  // Loss-driven K: replicas pause where an update starts in a new interval and K may still grow; each
+  // round schedules every replica up to its next pause (or the target), runs the arithmetic that far,
+  // evaluates the full-data risk and sets the paused replicas' new K.  Rounds = interval crossings + 1.
+  const bool adaptive = h->ada_loss;
+  if (adaptive) {
+    if (!h->F0_ready) { if ((st = eval_into(h, h->F0)) != SIM_OK) return st; h->F0_ready = true; }
+    sa.adaptive = 1; sa.target = h->n_updates + iters; sa.done = h->done; sa.run_j0 = h->run_j0; sa.run_iters = h->run_iters;
+    sa.K_cur = h->K_cur; sa.q_last = h->q_last; sa.want_eval = h->want_eval;
+  }
+  for (long long round = 0;; ++round) {
   schedule_kernel<<<(h->R + 3) / 4, 128, 0, h->stream>>>(sa);
   CUDA_TRY(h, cudaGetLastError());
 
   if (h->prob.model != SIM_NONE) {
     NumericArgs a{};
+    if (adaptive) { a.run_j0 = h->run_j0; a.run_iters = h->run_iters; }
     a.X = h->prob.X;
     a.y = h->prob.model == SIM_LSQ ? static_cast<const void*>(h->prob.y) : static_cast<const void*>(h->prob.label);
     a.w_ref = h->prob.w_ref; a.n = (uint64_t)h->prob.n; a.d = h->prob.d; a.m = h->m; a.model = (int)h->prob.model;
@@ -411,6 +456,19 @@ sim_status sim_run(sim_handle* h, int64_t iters) {
     }
     if (ce != cudaSuccess) st = fail(h, SIM_ERR_CUDA, std::string("numeric kernel launch: ") + cudaGetErrorString(ce));
     if (st != SIM_OK) { h->poisoned = true; return st; }
+  }
+  if (!adaptive) break;
+  if ((st = eval_into(h, h->Fcur)) != SIM_OK) { h->poisoned = true; return st; }
+  CUDA_TRY(h, cudaMemsetAsync(h->remaining, 0, sizeof(int), h->stream));
+  adasync_update_kernel<<<(h->R + 127) / 128, 128, 0, h->stream>>>(h->variant, h->P, h->K0, h->t_interval, h->R, sa.target, h->F0,
+                                                                  h->Fcur, h->clock, h->done, h->K_cur, h->q_last, h->want_eval,
+                                                                  h->remaining);
+  CUDA_TRY(h, cudaGetLastError());
+  int remaining = 0;
+  CUDA_TRY(h, cudaMemcpyAsync(&remaining, h->remaining, sizeof(int), cudaMemcpyDeviceToHost, h->stream));
+  CUDA_TRY(h, cudaStreamSynchronize(h->stream));
+  if (remaining == 0) break;
+  if (round > iters + 8) { h->poisoned = true; return fail(h, SIM_ERR_INTERNAL, "loss-driven K: no progress"); }
   }
   h->n_updates += iters;
   return SIM_OK;
@@ -469,25 +527,29 @@ sim_status sim_eval_loss(sim_handle* h, float* loss) {
   if (!h) return fail(nullptr, SIM_ERR_ARG, "handle is NULL");
   if (!loss) return fail(h, SIM_ERR_ARG, "loss is NULL");
   if (h->poisoned) return fail(h, SIM_ERR_STATE, "the handle failed earlier");
+  return eval_into(h, loss);
+}
+
+sim_status sim_set_adasync_loss(sim_handle* h, int32_t K0, double t_interval) {
+  if (!h) return fail(nullptr, SIM_ERR_ARG, "handle is NULL");
+  if (h->n_updates > 0 || h->cap > 0) return fail(h, SIM_ERR_STATE, "sim_set_adasync_loss is only allowed before sim_reserve / sim_run");
+  if (!(t_interval > 0.0)) return fail(h, SIM_ERR_ARG, "t_interval must be > 0");
+  if (K0 < 1 || K0 > h->P) return fail(h, SIM_ERR_ARG, "K0 must be in [1, P]");
   const sim_model mdl = h->prob.model;
   if (mdl != SIM_LSQ && mdl != SIM_LOGISTIC && mdl != SIM_SOFTMAX)
-    return fail(h, SIM_ERR_ARG, "sim_eval_loss is built for the linear models (LSQ, logistic, softmax)");
-  EvalArgs e{};
-  e.X = h->prob.X;
-  e.y = mdl == SIM_LSQ ? static_cast<const void*>(h->prob.y) : static_cast<const void*>(h->prob.label);
-  e.n = h->prob.n; e.d = h->prob.d; e.C = mdl == SIM_SOFTMAX ? h->prob.n_classes : 1; e.model = (int)mdl; e.R = h->R;
-  e.RB = EV_BN / e.C;
-  e.w_state = h->uses_pool ? nullptr : h->w_state;
-  e.pool = h->uses_pool ? h->pool : nullptr;
-  e.cur_slot = h->cur_slot; e.n_slots = h->n_slots; e.n_params = h->n_params; e.slot_stride = h->slot_stride;
-  e.row_blocks = (int)((h->prob.n + EV_BM - 1) / EV_BM);
-  if (!h->eval_partial) CUDA_TRY(h, dev_alloc(&h->eval_partial, (size_t)e.row_blocks * h->R, h->stream, false));
-  e.partial = h->eval_partial; e.out = loss;
-  dim3 grid((unsigned)e.row_blocks, (unsigned)((h->R + e.RB - 1) / e.RB));
-  eval_loss_kernel<<<grid, 256, 0, h->stream>>>(e);
+    return fail(h, SIM_ERR_ARG, "the loss-driven K rule needs the full-data risk: LSQ, logistic or softmax");
+  const size_t R = (size_t)h->R;
+  if (!h->F0) {
+    CUDA_TRY(h, dev_alloc(&h->F0, R, h->stream)); CUDA_TRY(h, dev_alloc(&h->Fcur, R, h->stream));
+    CUDA_TRY(h, dev_alloc(&h->done, R, h->stream)); CUDA_TRY(h, dev_alloc(&h->run_j0, R, h->stream));
+    CUDA_TRY(h, dev_alloc(&h->run_iters, R, h->stream)); CUDA_TRY(h, dev_alloc(&h->q_last, R, h->stream));
+    CUDA_TRY(h, dev_alloc(&h->K_cur, R, h->stream)); CUDA_TRY(h, dev_alloc(&h->want_eval, R, h->stream));
+    CUDA_TRY(h, dev_alloc(&h->remaining, 1, h->stream));
+  }
+  fill_int_kernel<<<(h->R + 127) / 128, 128, 0, h->stream>>>(h->K_cur, K0, h->R);
   CUDA_TRY(h, cudaGetLastError());
-  eval_loss_finish_kernel<<<(h->R + 127) / 128, 128, 0, h->stream>>>(e);
-  CUDA_TRY(h, cudaGetLastError());
+  h->ada_loss = true; h->F0_ready = false;
+  h->K0 = K0; h->t_interval = t_interval; h->K_stride = h->P;
   return SIM_OK;
 }
 

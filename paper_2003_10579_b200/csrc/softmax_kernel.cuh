@@ -51,6 +51,7 @@ __global__ void __launch_bounds__(SMX_NT) softmax_kernel(NumericArgs a) {
   const uint32_t rid = a.replica_base + (uint32_t)r;
   const uint32_t row_bytes = (uint32_t)d * 4u;
   const size_t np = (size_t)C * d;
+  const long long my_j0 = a.run_j0 ? a.run_j0[r] : a.j0, my_iters = a.run_iters ? a.run_iters[r] : a.iters;
 
   extern __shared__ __align__(128) unsigned char smem[];
   // fixed head (S <= 8), every array on a 16-byte boundary:
@@ -110,12 +111,12 @@ __global__ void __launch_bounds__(SMX_NT) softmax_kernel(NumericArgs a) {
     walk.advance(a);
   };
   if (warp == 0) {
-    walk.start(a, r);
+    walk.start(a, r, my_j0, my_iters);
     walk.tiles_per_task = (m + T - 1) / T;
     for (int s = 0; s < S; ++s) issue_tile(s);
   }
   __syncthreads();
-  if (a.iters <= 0) return;
+  if (my_iters <= 0) return;
 
   float G[CP][E];
 #pragma unroll
@@ -123,7 +124,7 @@ __global__ void __launch_bounds__(SMX_NT) softmax_kernel(NumericArgs a) {
 #pragma unroll
     for (int e = 0; e < E; ++e) G[c][e] = 0.f;
   float loss_acc = 0.f;      // meaningful in the row-leader threads (tid = 16 q)
-  long long j = a.j0;
+  long long j = my_j0;
   bool failed = false;
   // role in the softmax stage: 16 lanes per row
   const int sq = tid >> 4, sc = tid & 15;
