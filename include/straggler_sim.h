@@ -163,6 +163,15 @@ sim_status sim_get_params(const sim_handle* h, float* w);
  */
 sim_status sim_eval_loss(sim_handle* h, float* loss);
 
+/*
+ * Error against simulated wall clock on a common time grid - the error-runtime trade-off picture of
+ * Sections 1 and 5: for each grid time g (DEVICE array [n_grid]) the mean over replicas of the
+ * minibatch loss recorded at the replica's last update completed by g, and the number of replicas
+ * that have completed one by then (DEVICE outputs [n_grid]; mean 0 where the count is 0).
+ * Synchronises the handle's stream.  SIM_ERR_STATE before the first update.
+ */
+sim_status sim_error_curve(const sim_handle* h, const double* grid, int32_t n_grid, float* mean_loss, int32_t* count);
+
 /* Number of parameters of the handle's model (0 for SIM_NONE). */
 int64_t sim_n_params(const sim_handle* h);
 

@@ -6,6 +6,7 @@ the two share no code.
   core    Philox4x32-10, deterministic -ln(u), delays, minibatch indices, bulk arrival process (C)
   models  per-minibatch loss and gradient of the four models (numpy, fp64)
   sim     event-driven simulator of one replica (Python, interleaves arrivals and updates)
+  curves  error against wall clock on a common time grid
 """
-from . import core, models, sim  # noqa: F401
+from . import core, curves, models, sim  # noqa: F401
 from .sim import OracleReplica  # noqa: F401

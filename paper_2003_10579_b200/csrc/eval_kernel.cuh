@@ -133,4 +133,29 @@ __global__ void eval_loss_finish_kernel(EvalArgs a) {
   a.out[r] = (float)(s / (double)a.n);
 }
 
+// Error against simulated wall clock on a common time grid: at grid time g a replica contributes the
+// loss recorded at its last update with t <= g (binary search in its clock trace); the mean is over the
+// replicas that have completed an update by then.  One block per grid point, fp64 tree sum (fixed order).
+__global__ void __launch_bounds__(256) error_curve_kernel(const double* t, const float* err, long long cap, long long J, int R,
+                                                          const double* grid, float* mean, int* count) {
+  __shared__ double sum_s[256];
+  __shared__ int cnt_s[256];
+  const double g = grid[blockIdx.x];
+  double s = 0.0;
+  int c = 0;
+  for (int r = threadIdx.x; r < R; r += 256) {
+    const double* tr = t + (size_t)r * cap;
+    long long lo = 0, hi = J;                 // first index with t > g
+    while (lo < hi) { const long long mid = (lo + hi) >> 1; if (tr[mid] <= g) lo = mid + 1; else hi = mid; }
+    if (lo > 0) { s += (double)err[(size_t)r * cap + lo - 1]; ++c; }
+  }
+  sum_s[threadIdx.x] = s; cnt_s[threadIdx.x] = c;
+  __syncthreads();
+  for (int off = 128; off > 0; off >>= 1) {
+    if ((int)threadIdx.x < off) { sum_s[threadIdx.x] += sum_s[threadIdx.x + off]; cnt_s[threadIdx.x] += cnt_s[threadIdx.x + off]; }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) { count[blockIdx.x] = cnt_s[0]; mean[blockIdx.x] = cnt_s[0] ? (float)(sum_s[0] / cnt_s[0]) : 0.f; }
+}
+
 }  // namespace ssim

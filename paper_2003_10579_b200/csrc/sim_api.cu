@@ -553,6 +553,18 @@ sim_status sim_set_adasync_loss(sim_handle* h, int32_t K0, double t_interval) {
   return SIM_OK;
 }
 
+sim_status sim_error_curve(const sim_handle* h, const double* grid, int32_t n_grid, float* mean_loss, int32_t* count) {
+  if (!h) return fail(nullptr, SIM_ERR_ARG, "handle is NULL");
+  if (!grid || !mean_loss || !count || n_grid < 1) return fail(h, SIM_ERR_ARG, "grid, mean_loss, count and n_grid >= 1 are required");
+  sim_status st = device_error(h);
+  if (st != SIM_OK) return st;
+  if (h->n_updates == 0) return fail(h, SIM_ERR_STATE, "no updates have been simulated yet");
+  error_curve_kernel<<<n_grid, 256, 0, h->stream>>>(h->tr.t, h->tr.loss, h->cap, h->n_updates, h->R, grid, mean_loss, count);
+  CUDA_TRY(h, cudaGetLastError());
+  CUDA_TRY(h, cudaStreamSynchronize(h->stream));
+  return SIM_OK;
+}
+
 int64_t sim_n_params(const sim_handle* h) { return h ? h->n_params : 0; }
 
 const char* sim_last_error(const sim_handle* h) { return h ? h->last_error.c_str() : g_last_error.c_str(); }

@@ -43,3 +43,22 @@ def test_full_data_loss_is_refused_for_the_mlp():
         sim.eval_loss()
     assert e.value.status == 1
     sim.close()
+
+
+def test_error_curve_matches_the_oracle():
+    from oracle.curves import error_curve
+    from paper_2003_10579_b200 import binding as B
+    data = inputs.make_lsq(1000, 64, 0.1, 35)
+    sim = B.Simulation(to_device(data), P=8, K=3, variant="kasync", delay_kind="exp", mu=1.0, eta=0.02, m=8, seed=2, n_replicas=300)
+    with pytest.raises(B.SimError):
+        sim.error_curve([1.0])
+    sim.reserve(500)          # capacity larger than the updates done: the row pitch differs from J
+    sim.run(120)
+    tr = sim.trace()
+    grid = np.concatenate([[0.0, 1e-6], np.linspace(0.05, tr["t"].max() * 1.1, 40)])
+    mean, cnt = sim.error_curve(grid)
+    want_mean, want_cnt = error_curve(tr["t"], tr["loss"], grid)
+    assert np.array_equal(cnt, want_cnt)
+    assert np.allclose(mean, want_mean, rtol=1e-6, atol=0)
+    assert cnt[0] == 0 and cnt[-1] == 300 and mean[-1] < mean[5]
+    sim.close()

@@ -252,3 +252,13 @@ def test_ksync_order_statistics_under_pareto():
     tr = bulk("kbatchasync", 16, 4, "pareto2", 2.0, 1.0, seed=82, R=64, J=4000)
     rate = (tr["t"][:, -1] - tr["t"][:, 499]) / 3500
     assert abs(np.median(rate) - 4 * 2.0 / 16) < 0.05
+
+
+def test_error_curve_by_hand():
+    """Two replicas: at each grid time take the error of the last completed update, average those that have one."""
+    from oracle.curves import error_curve
+    t = np.array([[1.0, 2.0, 4.0], [0.5, 3.0, 3.5]])
+    e = np.array([[10.0, 8.0, 6.0], [20.0, 12.0, 4.0]])
+    mean, cnt = error_curve(t, e, [0.25, 0.5, 1.0, 2.5, 3.0, 10.0])
+    assert cnt.tolist() == [0, 1, 2, 2, 2, 2]
+    assert mean.tolist() == [0.0, 20.0, 15.0, 14.0, 10.0, 5.0]
