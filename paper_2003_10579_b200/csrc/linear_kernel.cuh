@@ -166,6 +166,7 @@ __global__ void __launch_bounds__(NT) linear1_kernel(NumericArgs a) {
   float* misc_s = red_s + 2 * NW * T;
   const size_t head = (size_t)((unsigned char*)(misc_s + NW) - smem);
   float* rows_s = reinterpret_cast<float*>(smem + ((head + 127) & ~(size_t)127));
+  uint32_t* pidx_s = reinterpret_cast<uint32_t*>(rows_s + (size_t)S * T * d);   // [m] sample rows of the producer's task
 
   if (tid == 0) {
     for (int s = 0; s < S; ++s) mbar_init(smem_addr(&full[s]), (uint32_t)T + 1u);
@@ -199,6 +200,15 @@ __global__ void __launch_bounds__(NT) linear1_kernel(NumericArgs a) {
     const int st = (int)(tile_no % S);
     const uint32_t bar = smem_addr(&full[st]);
     const int rows = min(T, m - walk.k * T);
+    if (walk.k == 0) {   // a new task: its m sample rows are drawn once, 32 at a time (only this warp uses the table)
+      __syncwarp();
+      for (int q = lane; q < m; q += 32) {
+        uint32_t idx = draw_index(a.seed, rid, walk.cur.worker, walk.cur.seq, (uint32_t)q, a.n);
+        if ((uint64_t)idx >= a.n) { atomicExch(a.err, ERR_BAD_INDEX); idx = 0; }
+        pidx_s[q] = idx;
+      }
+      __syncwarp();
+    }
     if (lane == 0) {
       TileInfo ti;
       ti.rows = rows; ti.K = (int)walk.cur.K; ti.snap = (int)walk.cur.snap; ti.fresh = (int)walk.cur.fresh;
@@ -213,9 +223,7 @@ __global__ void __launch_bounds__(NT) linear1_kernel(NumericArgs a) {
     __syncwarp();
     if (lane < T) {
       if (lane < rows) {
-        const uint32_t q = (uint32_t)(walk.k * T + lane);
-        uint32_t idx = draw_index(a.seed, rid, walk.cur.worker, walk.cur.seq, q, a.n);
-        if ((uint64_t)idx >= a.n) { atomicExch(a.err, ERR_BAD_INDEX); idx = 0; }
+        const uint32_t idx = pidx_s[walk.k * T + lane];
         bulk_g2s(smem_addr(rows_s + ((size_t)st * T + lane) * d), a.X + (size_t)idx * d, row_bytes, bar);
         word_g2s_arrive(smem_addr(&y_s[st * T + lane]), reinterpret_cast<const uint32_t*>(a.y) + idx, bar);
       } else {
@@ -389,10 +397,10 @@ __global__ void __launch_bounds__(NT) linear1_kernel(NumericArgs a) {
 }
 
 // shared-memory bytes of linear1_kernel for a given shape
-inline size_t linear1_smem_bytes(int NT, int T, int S, int d) {
+inline size_t linear1_smem_bytes(int NT, int T, int S, int d, int m) {
   size_t head = 8 * (size_t)S + sizeof(TileInfo) * (size_t)S + 4 * (size_t)S * T + 4 * (size_t)2 * (NT / 32) * T + 4 * (size_t)(NT / 32);
   head = (head + 127) & ~(size_t)127;
-  return head + (size_t)S * T * d * 4;
+  return head + (size_t)S * T * d * 4 + (size_t)m * 4;
 }
 
 }  // namespace ssim

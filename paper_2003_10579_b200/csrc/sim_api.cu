@@ -189,8 +189,8 @@ sim_status launch_linear1(sim_handle* h, NumericArgs& a) {
   }
   if (S < 2) S = 2;
   if (S > 8) S = 8;
-  size_t smem = linear1_smem_bytes(NT, T, S, d);
-  while (smem > (size_t)(226 << 10) && S > 2) { --S; smem = linear1_smem_bytes(NT, T, S, d); }
+  size_t smem = linear1_smem_bytes(NT, T, S, d, a.m);
+  while (smem > (size_t)(226 << 10) && S > 2) { --S; smem = linear1_smem_bytes(NT, T, S, d, a.m); }
   if (smem > (size_t)(226 << 10)) return fail(h, SIM_ERR_ARG, "d too large for the row staging buffers");
   a.stages = S;
   auto kern = a.is_async ? linear1_kernel<NT, CHUNKS, T, true> : linear1_kernel<NT, CHUNKS, T, false>;
@@ -300,7 +300,7 @@ sim_status sim_create(const sim_problem* problem, int32_t P, int32_t K, sim_vari
       if (prob.n_classes < 2 || prob.n_classes > SIM_MAX_CLASSES) return fail(nullptr, SIM_ERR_ARG, "n_classes must be in [2, SIM_MAX_CLASSES]");
     }
     if (prob.model == SIM_SOFTMAX) {
-      const char* why = softmax_shape_unsupported(prob.d, prob.n_classes);
+      const char* why = softmax_shape_unsupported(prob.d, prob.n_classes, m);
       if (why) return fail(nullptr, SIM_ERR_ARG, why);
     }
     if (prob.model == SIM_MLP2) {

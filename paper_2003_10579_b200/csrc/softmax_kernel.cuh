@@ -66,6 +66,7 @@ __global__ void __launch_bounds__(SMX_NT) softmax_kernel(NumericArgs a) {
   static_assert(64 + 4 * (T * 16 + NW * 64 + NW + T + 8 * T) + 8 * sizeof(TileInfo) <= SMX_HEAD_BYTES, "head too small");
   float* W_s = reinterpret_cast<float*>(smem + SMX_HEAD_BYTES);
   float* rows_s = W_s + np;
+  uint32_t* pidx_s = reinterpret_cast<uint32_t*>(rows_s + (size_t)S * T * d);   // [m] sample rows of the producer's task
 
   if (tid == 0) {
     for (int s = 0; s < S; ++s) mbar_init(smem_addr(&full[s]), (uint32_t)T + 1u);
@@ -85,6 +86,15 @@ __global__ void __launch_bounds__(SMX_NT) softmax_kernel(NumericArgs a) {
     const int st = (int)(tile_no % S);
     const uint32_t bar = smem_addr(&full[st]);
     const int rows = min(T, m - walk.k * T);
+    if (walk.k == 0) {   // a new task: its m sample rows are drawn once, 32 at a time (only this warp uses the table)
+      __syncwarp();
+      for (int q = lane; q < m; q += 32) {
+        uint32_t idx = draw_index(a.seed, rid, walk.cur.worker, walk.cur.seq, (uint32_t)q, a.n);
+        if ((uint64_t)idx >= a.n) { atomicExch(a.err, ERR_BAD_INDEX); idx = 0; }
+        pidx_s[q] = idx;
+      }
+      __syncwarp();
+    }
     if (lane == 0) {
       TileInfo ti;
       ti.rows = rows; ti.K = (int)walk.cur.K; ti.snap = (int)walk.cur.snap; ti.fresh = (int)walk.cur.fresh;
@@ -99,9 +109,7 @@ __global__ void __launch_bounds__(SMX_NT) softmax_kernel(NumericArgs a) {
     __syncwarp();
     if (lane < T) {
       if (lane < rows) {
-        const uint32_t q = (uint32_t)(walk.k * T + lane);
-        uint32_t idx = draw_index(a.seed, rid, walk.cur.worker, walk.cur.seq, q, a.n);
-        if ((uint64_t)idx >= a.n) { atomicExch(a.err, ERR_BAD_INDEX); idx = 0; }
+        const uint32_t idx = pidx_s[walk.k * T + lane];
         bulk_g2s(smem_addr(rows_s + ((size_t)st * T + lane) * d), a.X + (size_t)idx * d, row_bytes, bar);
         word_g2s_arrive(smem_addr(&y_s[st * T + lane]), reinterpret_cast<const uint32_t*>(a.y) + idx, bar);
       } else {
@@ -123,11 +131,12 @@ __global__ void __launch_bounds__(SMX_NT) softmax_kernel(NumericArgs a) {
   for (int c = 0; c < CP; ++c)
 #pragma unroll
     for (int e = 0; e < E; ++e) G[c][e] = 0.f;
-  float loss_acc = 0.f;      // meaningful in the row-leader threads (tid = 16 q)
+  float loss_acc = 0.f;      // meaningful in the row-leader threads of the softmax stage
   long long j = my_j0;
   bool failed = false;
   // role in the softmax stage: 16 lanes per row
-  const int sq = tid >> 4, sc = tid & 15;
+  const int st_tid = tid - (NT - 16 * T);          // the last two warps serve the softmax stage (warp 0 is the producer)
+  const int sq = st_tid >> 4, sc = st_tid & 15;
 
   for (long long it = 0;; ++it) {
     const int st = (int)(it % S);
@@ -155,7 +164,7 @@ __global__ void __launch_bounds__(SMX_NT) softmax_kernel(NumericArgs a) {
       }
     }
     int label = 0;
-    if (tid < 16 * T && sq < ti.rows) label = (int)y_s[st * T + sq];
+    if (st_tid >= 0 && sq < ti.rows) label = (int)y_s[st * T + sq];
 
     // ---- Z partials over own columns, one half of the classes at a time ----
 #pragma unroll
@@ -192,7 +201,7 @@ __global__ void __launch_bounds__(SMX_NT) softmax_kernel(NumericArgs a) {
     if (warp == 0) issue_tile(it + S);
 
     // ---- softmax stage: thread (sq, sc) owns logit (row sq, class sc) ----
-    if (tid < 16 * T) {
+    if (st_tid >= 0) {
       float z = -INFINITY;
       const bool live = sc < C && sq < ti.rows;
       if (live) {
@@ -278,7 +287,7 @@ __global__ void __launch_bounds__(SMX_NT) softmax_kernel(NumericArgs a) {
       if (ASYNC) cur_slot = ti.fresh;
       dd = warp_sum(dd);
       if (lane == 0) misc_s[warp] = dd;
-      if (tid < 16 * T && sc == 0) lossrow_s[sq] = loss_acc;
+      if (st_tid >= 0 && sc == 0) lossrow_s[sq] = loss_acc;
       __syncthreads();   // (C)
       if (tid == 0) {
         float tot = 0.f, ls = 0.f;
@@ -304,15 +313,15 @@ __global__ void __launch_bounds__(SMX_NT) softmax_kernel(NumericArgs a) {
   }
 }
 
-inline size_t softmax_smem_bytes(int S, int d, int C) {
-  return (size_t)SMX_HEAD_BYTES + (size_t)C * d * 4 + (size_t)S * SMX_T * d * 4;
+inline size_t softmax_smem_bytes(int S, int d, int C, int m) {
+  return (size_t)SMX_HEAD_BYTES + (size_t)C * d * 4 + (size_t)S * SMX_T * d * 4 + (size_t)m * 4;
 }
 
-inline const char* softmax_shape_unsupported(int d, int C) {
+inline const char* softmax_shape_unsupported(int d, int C, int m) {
   const int d4 = d / 4;
   if (C <= 10 && d4 > 2 * SMX_NT) return "softmax: d > 3072 is not supported for up to 10 classes";
   if (C > 10 && d4 > SMX_NT) return "softmax: d > 1536 is not supported for more than 10 classes";
-  if (softmax_smem_bytes(2, d, C) > (size_t)(226 << 10)) return "softmax: W and two row tiles do not fit in shared memory";
+  if (softmax_smem_bytes(2, d, C, m) > (size_t)(226 << 10)) return "softmax: W and two row tiles do not fit in shared memory";
   return nullptr;
 }
 
@@ -326,11 +335,11 @@ cudaError_t launch_softmax(NumericArgs& a, int S, size_t smem, cudaStream_t stre
 }
 
 inline cudaError_t run_softmax(NumericArgs& a, int tune_stages, cudaStream_t stream, const char** why) {
-  *why = softmax_shape_unsupported(a.d, a.n_classes);
+  *why = softmax_shape_unsupported(a.d, a.n_classes, a.m);
   if (*why) return cudaSuccess;
   int S = tune_stages > 0 ? tune_stages : 8;
-  while (S > 2 && softmax_smem_bytes(S, a.d, a.n_classes) > (size_t)(226 << 10)) --S;
-  const size_t smem = softmax_smem_bytes(S, a.d, a.n_classes);
+  while (S > 2 && softmax_smem_bytes(S, a.d, a.n_classes, a.m) > (size_t)(226 << 10)) --S;
+  const size_t smem = softmax_smem_bytes(S, a.d, a.n_classes, a.m);
   a.stages = S;
   const int d4 = a.d / 4;
   if (a.n_classes <= 10) return d4 <= SMX_NT ? launch_softmax<1, 10>(a, S, smem, stream) : launch_softmax<2, 10>(a, S, smem, stream);
