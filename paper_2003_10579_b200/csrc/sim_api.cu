@@ -205,7 +205,11 @@ sim_status run_linear1(sim_handle* h, NumericArgs& a) {
   if (d4 <= 32) return launch_linear1<32, 1, 8>(h, a);
   if (d4 <= 64) return launch_linear1<64, 1, 8>(h, a);
   if (d4 <= 128) return launch_linear1<128, 1, 4>(h, a);
-  if (d4 <= 256) return launch_linear1<128, 2, 4>(h, a);
+  if (d4 <= 256) {
+    const int rows = h->tune_rows ? h->tune_rows : 4;
+    if (h->tune_threads == 256) return rows == 8 ? launch_linear1<256, 1, 8>(h, a) : launch_linear1<256, 1, 4>(h, a);
+    return rows == 8 ? launch_linear1<128, 2, 8>(h, a) : rows == 2 ? launch_linear1<128, 2, 2>(h, a) : launch_linear1<128, 2, 4>(h, a);
+  }
   if (d4 <= 512) return launch_linear1<256, 2, 4>(h, a);
   if (d4 <= 1024) {
     const int rows = h->tune_rows ? h->tune_rows : (a.R > 148 ? 2 : 4), threads = h->tune_threads ? h->tune_threads : 256;
@@ -378,7 +382,7 @@ sim_status sim_set_adasync(sim_handle* h, int32_t K0, double t_interval) {
 sim_status sim_set_tuning(sim_handle* h, int32_t stages, int32_t tile_rows, int32_t threads) {
   if (!h) return fail(nullptr, SIM_ERR_ARG, "handle is NULL");
   if (stages < 0 || stages == 1 || stages > 8) return fail(h, SIM_ERR_ARG, "stages must be 0 (automatic) or in [2, 8]");
-  if (tile_rows != 0 && tile_rows != 2 && tile_rows != 4) return fail(h, SIM_ERR_ARG, "tile_rows must be 0, 2 or 4");
+  if (tile_rows != 0 && tile_rows != 2 && tile_rows != 4 && tile_rows != 8) return fail(h, SIM_ERR_ARG, "tile_rows must be 0, 2, 4 or 8");
   if (threads != 0 && threads != 256 && threads != 512) return fail(h, SIM_ERR_ARG, "threads must be 0, 256 or 512");
   h->tune_stages = stages; h->tune_rows = tile_rows; h->tune_threads = threads;
   return SIM_OK;
