@@ -1,0 +1,71 @@
+"""GPU parity at the degenerate ends of the parameter ranges: one sample, one feature block, one
+worker, minibatch of one, 32 workers with K = 32, replica ids at the top of the 32-bit range, a single
+replica, and zero-length / repeated runs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import core
+from paper_2003_10579_b200 import inputs
+from parity import assert_schedule_equal, to_device
+from test_gpu_linear import run_case
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2003_10579_b200 import binding
+    return binding
+
+
+@pytest.mark.parametrize("variant", list(core.VARIANTS))
+def test_smallest_shapes(B, variant):
+    run_case(B, inputs.make_lsq(1, 4, 0.0, 50), variant=variant, P=1, K=1, m=1, eta=0.05, R=1, J=12, chunks=[3])     # one sample
+    run_case(B, inputs.make_lsq(7, 4, 0.1, 51), variant=variant, P=3, K=2, m=1, eta=0.05, R=2, J=15, chunks=[4])
+    run_case(B, inputs.make_logistic(33, 8, 0.1, 52), variant=variant, P=2, K=2, m=3, eta=0.1, R=3, J=15, use_ref=False)
+    run_case(B, inputs.make_mixture(40, 4, 2, 0.5, 53), variant=variant, P=2, K=1, m=5, eta=0.1, R=2, J=12, use_ref=False)
+
+
+@pytest.mark.parametrize("variant", list(core.VARIANTS))
+def test_all_32_workers_contribute(B, variant):
+    run_case(B, inputs.make_lsq(500, 32, 0.1, 54), variant=variant, P=32, K=32, m=2, eta=0.05, R=3, J=10, chunks=[2])
+
+
+def test_replica_ids_at_the_top_of_the_range(B):
+    base = 2**32 - 5
+    run_case(B, inputs.make_lsq(300, 16, 0.1, 55), variant="kbatchasync", P=4, K=2, m=4, eta=0.05, R=5, J=20, base=base)
+    sim = B.Simulation(None, P=4, K=2, variant="kasync", delay_kind="exp", mu=1.0, eta=0.0, m=1, seed=7, n_replicas=5, replica_base=base)
+    sim.run(40)
+    ora = core.BulkSchedule("kasync", 4, 2, "exp", 1.0, 0.0, 7, 5, replica_base=base).run(40)
+    assert_schedule_equal(sim.trace(), ora)
+    sim.close()
+
+
+def test_zero_length_and_many_short_runs(B):
+    data = inputs.make_lsq(200, 16, 0.1, 56)
+    dev = to_device(data)
+    kw = dict(P=4, K=2, variant="kasync", delay_kind="exp", mu=1.0, eta=0.05, m=4, seed=3, n_replicas=4)
+    a, b = B.Simulation(dev, **kw), B.Simulation(dev, **kw)
+    assert a.trace_size()[0] == 0 and a.trace()["t"].shape == (4, 0)
+    a.run(0)
+    a.run(30)
+    for _ in range(30):
+        b.run(1)           # thirty growths of the trace from capacity 1
+    ta, tb = a.trace(), b.trace()
+    for k in ta:
+        assert np.array_equal(ta[k], tb[k]), k
+    assert np.array_equal(a.params(), b.params())
+    a.close(); b.close()
+
+
+def test_seed_uses_all_64_bits(B):
+    kw = dict(P=4, K=2, variant="ksync", delay_kind="exp", mu=1.0, eta=0.0, m=1, n_replicas=2)
+    out = []
+    for seed in (1, 1 + 2**32, 2**63 + 1):
+        sim = B.Simulation(None, seed=seed, **kw)
+        sim.run(5)
+        out.append(sim.trace()["t"])
+        assert_schedule_equal(sim.trace(), core.BulkSchedule("ksync", 4, 2, "exp", 1.0, 0.0, seed, 2).run(5))
+        sim.close()
+    assert not np.array_equal(out[0], out[1]) and not np.array_equal(out[0], out[2])
