@@ -28,7 +28,9 @@ namespace ssim {
 
 struct MlpScratch {
   __nv_bfloat16* Xq = nullptr;     // [n][d]                   bf16 copy of the data set
-  __nv_bfloat16* W1qT = nullptr;   // [R][n_slots][H][d]       bf16 shadow of every W1 version, transposed (d contiguous)
+  __nv_bfloat16* W1qT = nullptr;   // [R][n_slots][d/64][H][64] bf16 shadow of every W1 version, transposed and tiled: the
+                                   //                          64 k-values of a k-block are contiguous per hidden unit, so the
+                                   //                          [H x 64] operand tile of one k-block is one contiguous block
   __nv_bfloat16* D1q = nullptr;    // [R][Kmax][m][H]          bf16(delta1) of the current update
   float* Hact = nullptr;           // [R][Kmax][m][H]          h
   float* D2 = nullptr;             // [R][Kmax][m][16]         delta2
@@ -84,13 +86,15 @@ __global__ void to_bf16_kernel(const float* src, __nv_bfloat16* dst, long long c
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < count; i += (long long)gridDim.x * blockDim.x)
     dst[i] = __float2bfloat16_rn(src[i]);
 }
-// transposed bf16 shadow (W1^T [H][d]) of W1 in pool slot `slot` of every replica
+// transposed, k-block-tiled bf16 shadow of W1 in pool slot `slot` of every replica:
+// element (k, n) of W1 goes to [(k / 64) * H + n] * 64 + k % 64
 __global__ void shadow_w1_kernel(const float* pool, __nv_bfloat16* W1qT, long long slot_stride, int d, int H, int n_slots, int slot, int R) {
   const long long dH = (long long)d * H, total = dH * R;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
     const long long r = i / dH, p = i % dH;
-    const long long n = p / d, k = p % d;       // output element (n, k) = W1[k][n]
-    W1qT[((size_t)r * n_slots + slot) * dH + p] = __float2bfloat16_rn(pool[((size_t)r * n_slots + slot) * slot_stride + k * H + n]);
+    const long long kb = p / (64ll * H), n = (p / 64) % H, kk = p % 64;
+    W1qT[((size_t)r * n_slots + slot) * dH + p] =
+        __float2bfloat16_rn(pool[((size_t)r * n_slots + slot) * slot_stride + (kb * 64 + kk) * H + n]);
   }
 }
 

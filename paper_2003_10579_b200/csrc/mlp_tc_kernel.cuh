@@ -2,8 +2,9 @@
 // memory.
 //
 // One CTA per (replica, contributor, 128-sample block):  A1[128 x H] = bf16(X_b)[128 x d] bf16(W1)[d x H]
-//   warp 0   B producer: TMA tensor loads of the W1 tile from the transposed bf16 shadow W1^T [H][d]
-//            (K-major B operand, 128-byte swizzle, one or two boxes per stage)
+//   warp 0   B producer: TMA tensor loads of the W1 tile from the transposed, k-block-tiled bf16 shadow
+//            (K-major B operand, 128-byte swizzle; a stage's [H x 64] tile is one contiguous block of the
+//            shadow, fetched as one or two boxes)
 //   warps 2-5  A producer during the main loop: the 128 gathered sample rows of a stage are 1024
 //            16-byte pieces, copied with cp.async into the same 128-byte-swizzle pattern (one-row
 //            TMA boxes of 128 B were limited by the TMA instruction rate), made visible to the
@@ -168,7 +169,7 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
 
   if (warp == 0) {
     // ---- B producer ----
-    const int w_row0 = (int)(((size_t)r * sc.n_slots + snap) * H);
+    const long long w_blk0 = ((long long)r * sc.n_slots + snap) * (d / TC_BK);     // first k-block of this W1^T shadow
     if (lane == 0) {
       for (int kc = 0; kc < nk; ++kc) {
         const int s = kc % S;
@@ -176,7 +177,7 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
         const uint32_t Bs = base_addr + (uint32_t)s * L.stage_bytes + TC_A_BYTES;
         mbar_arrive_expect_tx(full_bar(s), (uint32_t)(H * 128));
         for (int hf = 0; hf < n_halves; ++hf)
-          tma_load_2d(Bs + (uint32_t)hf * n_inst * 128, &tmW, kc * TC_BK, w_row0 + hf * n_inst, full_bar(s));
+          tma_load_2d(Bs + (uint32_t)hf * n_inst * 128, &tmW, 0, (int)((w_blk0 + kc) * H + hf * n_inst), full_bar(s));
       }
     }
     __syncwarp();
@@ -522,7 +523,8 @@ mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
       const float scale = (float)((double)a.eta / ((double)K * (double)m));
       const float* wc = tile_ptr(t);
       float* wn = a.pool + ((size_t)r * a.n_slots + fresh) * a.slot_stride + row * H + col0;
-      __nv_bfloat16* wq = sc.W1qT + ((size_t)r * sc.n_slots + fresh) * dH + (size_t)col0 * d + row;   // [H][d]
+      // shadow element (k = row, n) lives at [(row / 64) * H + n] * 64 + row % 64
+      __nv_bfloat16* wq = sc.W1qT + ((size_t)r * sc.n_slots + fresh) * dH + ((size_t)(row >> 6) * H + col0) * 64 + (row & 63);
       if (t + (int)gridDim.x < n_tiles) {            // the next tile's w_j: ask L2 for it a whole tile ahead
         const float* pn = tile_ptr(t + gridDim.x);
         for (int c = 0; c < nch; ++c) prefetch_l2(pn + c * 32);
@@ -552,10 +554,10 @@ mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
           w.w = fmaf(-scale, __uint_as_float(v[4 * i4 + 3]), w.w);
           reinterpret_cast<float4*>(wn + ch * 32)[i4] = w;
           const int col = ch * 32 + 4 * i4;
-          wq[(size_t)col * d] = __float2bfloat16_rn(w.x);
-          wq[(size_t)(col + 1) * d] = __float2bfloat16_rn(w.y);
-          wq[(size_t)(col + 2) * d] = __float2bfloat16_rn(w.z);
-          wq[(size_t)(col + 3) * d] = __float2bfloat16_rn(w.w);
+          wq[(size_t)col * 64] = __float2bfloat16_rn(w.x);
+          wq[(size_t)(col + 1) * 64] = __float2bfloat16_rn(w.y);
+          wq[(size_t)(col + 2) * 64] = __float2bfloat16_rn(w.z);
+          wq[(size_t)(col + 3) * 64] = __float2bfloat16_rn(w.w);
         }
       }
       tc_fence_before();                 // this warp's reads of the buffer are done: hand it back
@@ -606,7 +608,7 @@ inline cudaError_t run_mlp(NumericArgs& a, MlpScratch& s, MlpMaps& maps, int P, 
   const int n_halves = s.H > 256 ? 2 : 1;
   if (!maps.ready) {
     if (!tc_make_map(&maps.tmX, s.Xq, (uint64_t)s.n, (uint64_t)s.d, TC_BK, 1) ||
-        !tc_make_map(&maps.tmW, s.W1qT, (uint64_t)s.R * s.n_slots * s.H, (uint64_t)s.d, TC_BK, (uint32_t)(s.H / n_halves)) ||
+        !tc_make_map(&maps.tmW, s.W1qT, (uint64_t)s.R * s.n_slots * (s.d / TC_BK) * s.H, (uint64_t)TC_BK, TC_BK, (uint32_t)(s.H / n_halves)) ||
         !tc_make_map(&maps.tmD, s.D1q, (uint64_t)s.R * s.Kmax * s.m, (uint64_t)s.H, 64, 64)) {
       *why = "mlp: could not encode the TMA tensor maps";
       return cudaSuccess;
