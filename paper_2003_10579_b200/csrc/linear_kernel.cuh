@@ -51,6 +51,16 @@ struct NumericArgs {
   int* err;
 };
 
+// Where the MLP keeps element (k, n) of W1 inside a version of the pool.  The update kernel moves W1
+// one 128-row x 32-column block at a time; stored block by block - [d/128][H/32][128][32] - a block is
+// 16 KB contiguous (one bulk copy each way), a tile of the kernel a contiguous run of blocks.  Inside a
+// row of a block the eight 16-byte pieces are XOR-swizzled with the row number, so that a thread per row
+// reads its row from shared memory without bank conflicts.  Callers see the row-major order:
+// sim_set_params / sim_get_params convert.
+__host__ __device__ __forceinline__ long long w1_tiled_index(long long k, long long n, int H) {
+  return (((k >> 7) * (H >> 5) + (n >> 5)) << 12) + ((k & 127) << 5) + (((((n & 31) >> 2) ^ (k & 7)) << 2) | (n & 3));
+}
+
 // ---- shared-memory barrier and bulk-copy primitives ------------------------------------------
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 

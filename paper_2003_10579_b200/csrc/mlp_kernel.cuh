@@ -1,7 +1,7 @@
 // Two-layer relu MLP (d - H - C, softmax cross-entropy) under the simulated schedule.
 //
-// Parameters per version: [W1 (d x H row-major), b1 (H), W2 (H x C row-major), b2 (C)], fp32,
-// kept in a pool of immutable versions per replica, plus a bf16 shadow of W1 per version and a
+// Parameters per version: [W1 (d x H), b1 (H), W2 (H x C row-major), b2 (C)], fp32, kept in a pool of
+// immutable versions per replica (W1 block-tiled inside the pool, see w1_tiled_index; row-major to callers), plus a bf16 shadow of W1 per version and a
 // bf16 copy of the data set.  The two products over d take bf16 operands and accumulate in fp32
 // on the tensor cores:
 //     A1 = bf16(X_b) bf16(W1)          (forward,  [m x d] [d x H])
@@ -94,7 +94,7 @@ __global__ void shadow_w1_kernel(const float* pool, __nv_bfloat16* W1qT, long lo
     const long long r = i / dH, p = i % dH;
     const long long kb = p / (64ll * H), n = (p / 64) % H, kk = p % 64;
     W1qT[((size_t)r * n_slots + slot) * dH + p] =
-        __float2bfloat16_rn(pool[((size_t)r * n_slots + slot) * slot_stride + (kb * 64 + kk) * H + n]);
+        __float2bfloat16_rn(pool[((size_t)r * n_slots + slot) * slot_stride + w1_tiled_index(kb * 64 + kk, n, H)]);
   }
 }
 

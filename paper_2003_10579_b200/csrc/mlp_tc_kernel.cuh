@@ -353,16 +353,21 @@ __device__ __forceinline__ uint64_t tc_desc_mnmajor(uint32_t saddr, uint32_t lbo
 
 // ---- dW1 = bf16(X)^T bf16(delta1), fused with the update of W1: persistent kernel -----------------
 // Tiles of 128 rows of W1 x Hn columns (Hn <= 256) are dealt round-robin to one CTA per SM.  The
-// accumulator is double-buffered in tensor memory, so the row-per-thread epilogue of one tile
-// (read w_j, apply Eq. 2 / Eq. 3, write w_{j+1} and its transposed bf16 shadow) overlaps the loads
-// and MMAs of the next.  Both operands are MN-major and used exactly as stored: a stage holds 64
-// samples; A = their features [slab*128, +128) gathered from the bf16 data set (cp.async by four
-// producer warps into the 128-byte-swizzle atom layout), B = the same samples' bf16 delta1 columns
-// (TMA boxes of 64 x 64).  dW1 itself never exists in memory.
+// accumulator is double-buffered in tensor memory, so the epilogue of one tile overlaps the loads and
+// MMAs of the next.  Both operands are MN-major and used exactly as stored: a stage holds 64 samples;
+// A = their features [slab*128, +128) gathered from the bf16 data set (cp.async by four producer warps
+// into the 128-byte-swizzle atom layout), B = the same samples' bf16 delta1 columns (TMA boxes of
+// 64 x 64).  dW1 itself never exists in memory.
+// The epilogue never touches global memory from a register: w_j streams in as 16 KB blocks (128 rows x 32
+// columns, contiguous in the pool) by bulk copies into a ring of shared-memory slots, a group of four
+// warps (thread = row) applies Eq. 2 / Eq. 3 in place from the accumulator, writes the bf16 shadow of the
+// block beside it, and one thread sends both out with bulk stores.
 //   warp 0      TMA producer of B          warp 1      tcgen05.mma issuer, owns tensor memory
-//   warps 2-5   cp.async producers of A    warps 6-13  epilogue (one row of W1 per thread, two warps per
-//                                                      tensor-memory lane quarter, half of the columns each)
-constexpr int DW1_THREADS = 448;
+//   warps 2-5   cp.async producers of A    warps 6-13  epilogue: two groups of four warps (one per tensor-
+//   warp 14     bulk-copy producer of w_j               memory lane quarter), blocks of a tile dealt alternately
+constexpr int DW1_THREADS = 480;
+constexpr int DW1_WBLOCK = 16384;        // one block of W1 in fp32
+constexpr int DW1_QSTAGE = 8192;         // its bf16 shadow: two k-blocks of 32 columns x 64 rows
 
 // columns per tile: the largest H/p that is at most 256 and a multiple of 64
 inline __host__ __device__ int tc_dw1_cols(int H) {
@@ -370,17 +375,34 @@ inline __host__ __device__ int tc_dw1_cols(int H) {
     if (H % p == 0 && H / p <= 256 && (H / p) % 64 == 0) return H / p;
   return 64;
 }
-struct TcDw1Layout { int stages, stage_bytes, off_bars, off_tmem, total; };
+struct TcDw1Layout { int stages, stage_bytes, wslots, off_w, off_q, off_bars, off_tmem, off_fail, total; };
 inline __host__ __device__ TcDw1Layout tc_dw1_layout(int H) {
   TcDw1Layout L;
+  const int budget = 224 << 10;
   L.stage_bytes = TC_A_BYTES + tc_dw1_cols(H) * 128;     // A: 64 samples x 128 features; B: 64 samples x Hn
-  L.stages = (200 << 10) / L.stage_bytes;
+  L.stages = (budget - 2 * DW1_QSTAGE - 3 * DW1_WBLOCK) / L.stage_bytes;
   if (L.stages > 4) L.stages = 4;
-  L.off_bars = L.stages * L.stage_bytes;
-  L.off_tmem = L.off_bars + 8 * (2 * L.stages + 4);
-  L.total = L.off_tmem + 16 + 1024;
+  L.wslots = (budget - 2 * DW1_QSTAGE - L.stages * L.stage_bytes) / DW1_WBLOCK;
+  if (L.wslots > 6) L.wslots = 6;
+  L.off_w = L.stages * L.stage_bytes;
+  L.off_q = L.off_w + L.wslots * DW1_WBLOCK;
+  L.off_bars = L.off_q + 2 * DW1_QSTAGE;
+  L.off_tmem = L.off_bars + 8 * (2 * L.stages + 4 + 2 * L.wslots);
+  L.off_fail = L.off_tmem + 16;
+  L.total = L.off_fail + 16 + 1024;
   return L;
 }
+
+__device__ __forceinline__ void bulk_s2g(void* dst, uint32_t src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void group_barrier(int id, int threads) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory"); }
 
 __global__ void __launch_bounds__(DW1_THREADS, 1)
 mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
@@ -402,16 +424,22 @@ mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
   unsigned char* base = smem_raw + (base_addr - raw_addr);
   const TcDw1Layout L = tc_dw1_layout(H);
   const int S = L.stages;
-  const uint32_t bars = base_addr + L.off_bars;     // full[S] | empty[S] | acc_full[2] | acc_empty[2]
+  const int NB = L.wslots;
+  const uint32_t bars = base_addr + L.off_bars;     // full[S] | empty[S] | acc_full[2] | acc_empty[2] | wfull[NB] | wempty[NB]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base + L.off_tmem);
+  volatile int* fail_s = reinterpret_cast<volatile int*>(base + L.off_fail);     // one flag per epilogue group
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (S + s); };
   auto acc_full = [&](int b) { return bars + 8u * (2 * S + b); };
   auto acc_empty = [&](int b) { return bars + 8u * (2 * S + 2 + b); };
+  auto wfull = [&](int s) { return bars + 8u * (2 * S + 4 + s); };
+  auto wempty = [&](int s) { return bars + 8u * (2 * S + 4 + NB + s); };
 
   if (tid == 0) {
     for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1 + 128); mbar_init(empty_bar(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 8); }
+    for (int s = 0; s < NB; ++s) { mbar_init(wfull(s), 1); mbar_init(wempty(s), 1); }
+    fail_s[0] = 0; fail_s[1] = 0;
     mbar_fence_init();
   }
   if (warp == 1) tc_alloc(smem_addr(tmem_slot), tmem_cols);
@@ -503,67 +531,88 @@ mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
     }
     cp_async_wait<0>();
     if (!failed) while (signalled < it) signal(signalled++);
-  } else {
-    // ---- epilogue: thread = one row of W1 of the tile, columns [half*Hn/2, +Hn/2) ----
-    const int q = warp & 3;             // the tensor-memory lane quarter this warp may read
-    const int half = (warp - 6) >> 2, Hh = Hn / 2, nch = Hh / 32;
-    auto tile_ptr = [&](int t) {        // this thread's part of w_j in tile t
-      const int r = tile_r(t), slab = (t / parts) % slabs, part = t % parts;
-      return a.pool + ((size_t)r * a.n_slots + mlp_cur_slot(a, r, j)) * a.slot_stride +
-             ((size_t)slab * 128 + 32 * q + lane) * H + part * Hn + half * Hh;
-    };
+  } else if (warp < 14) {
+    // ---- epilogue: thread = one row of the 128-row block; group grp takes blocks grp, grp + 2, ... of a tile ----
+    const int q = warp & 3, grp = (warp - 6) >> 2;      // q: the tensor-memory lane quarter this warp may read
+    const int rloc = 32 * q + lane, nb = Hn / 32;
+    const bool leader = ((warp - 6) & 3) == 0 && lane == 0;
+    unsigned char* qstage = base + L.off_q + grp * DW1_QSTAGE;
+    // shadow element (k, n) lives at [(k / 64) * H + n] * 64 + k % 64: in the staging copy of a block,
+    // [k / 64][n - first column][k % 64]
+    __nv_bfloat16* qrow = reinterpret_cast<__nv_bfloat16*>(qstage) + (rloc >> 6) * 2048 + (rloc & 63);
+    long long n = grp;                                  // running number of the block among all blocks of this CTA
     int i = 0;
-    if ((int)blockIdx.x < n_tiles) { const float* p0 = tile_ptr(blockIdx.x); for (int c = 0; c < nch; ++c) prefetch_l2(p0 + c * 32); }
     for (int t = blockIdx.x; t < n_tiles && !failed; t += gridDim.x, ++i) {
       const int r = tile_r(t), slab = (t / parts) % slabs, part = t % parts, buf = i & 1;
       const int K = (int)a.K_used[(size_t)r * a.cap + j];
-      const size_t row = (size_t)slab * 128 + 32 * q + lane;
-      const int col0 = part * Hn + half * Hh;
       const int fresh = mlp_fresh_slot(a, r, j);
       const float scale = (float)((double)a.eta / ((double)K * (double)m));
-      const float* wc = tile_ptr(t);
-      float* wn = a.pool + ((size_t)r * a.n_slots + fresh) * a.slot_stride + row * H + col0;
-      // shadow element (k = row, n) lives at [(row / 64) * H + n] * 64 + row % 64
-      __nv_bfloat16* wq = sc.W1qT + ((size_t)r * sc.n_slots + fresh) * dH + ((size_t)(row >> 6) * H + col0) * 64 + (row & 63);
-      if (t + (int)gridDim.x < n_tiles) {            // the next tile's w_j: ask L2 for it a whole tile ahead
-        const float* pn = tile_ptr(t + gridDim.x);
-        for (int c = 0; c < nch; ++c) prefetch_l2(pn + c * 32);
-      }
-      float4 wnext[8];                                // w_j of the chunk after the one being processed
-#pragma unroll
-      for (int i4 = 0; i4 < 8; ++i4) wnext[i4] = reinterpret_cast<const float4*>(wc)[i4];
-      if (!mbar_wait(acc_full(buf), (uint32_t)((i >> 1) & 1))) { failed = true; break; }
-      tc_fence_after();
-      const uint32_t trow = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * Hn + half * Hh);
-      uint32_t v[32];
-      for (int ch = 0; ch < nch; ++ch) {
-        float4 wcur[8];
-#pragma unroll
-        for (int i4 = 0; i4 < 8; ++i4) wcur[i4] = wnext[i4];
-        if (ch + 1 < nch) {
-#pragma unroll
-          for (int i4 = 0; i4 < 8; ++i4) wnext[i4] = reinterpret_cast<const float4*>(wc + (ch + 1) * 32)[i4];
-        }
-        tc_ld32(trow + ch * 32, v);
+      float* wn = a.pool + ((size_t)r * a.n_slots + fresh) * a.slot_stride + (((size_t)slab * (H >> 5) + ((part * Hn) >> 5)) << 12);
+      __nv_bfloat16* wq = sc.W1qT + ((size_t)r * sc.n_slots + fresh) * dH + ((size_t)(2 * slab) * H + part * Hn) * 64;
+      const uint32_t trow = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * Hn);
+      for (int b = grp; b < nb; b += 2, n += 2) {
+        const int s = (int)(n % NB);
+        bool ok = mbar_wait(wfull(s), (uint32_t)((n / NB) & 1));
+        if (ok && b == grp) ok = mbar_wait(acc_full(buf), (uint32_t)((i >> 1) & 1));
+        if (!ok) fail_s[grp] = 1;
+        group_barrier(1 + grp, 128);                    // the four warps give up together or not at all
+        if (fail_s[grp]) { failed = true; break; }
+        tc_fence_after();
+        uint32_t v[32];
+        tc_ld32(trow + b * 32, v);
+        float4* wrow = reinterpret_cast<float4*>(base + L.off_w + s * DW1_WBLOCK + rloc * 128);
 #pragma unroll
         for (int i4 = 0; i4 < 8; ++i4) {
-          float4 w = wcur[i4];
+          float4 w = wrow[i4 ^ (rloc & 7)];
           w.x = fmaf(-scale, __uint_as_float(v[4 * i4]), w.x);
           w.y = fmaf(-scale, __uint_as_float(v[4 * i4 + 1]), w.y);
           w.z = fmaf(-scale, __uint_as_float(v[4 * i4 + 2]), w.z);
           w.w = fmaf(-scale, __uint_as_float(v[4 * i4 + 3]), w.w);
-          reinterpret_cast<float4*>(wn + ch * 32)[i4] = w;
-          const int col = ch * 32 + 4 * i4;
-          wq[(size_t)col * 64] = __float2bfloat16_rn(w.x);
-          wq[(size_t)(col + 1) * 64] = __float2bfloat16_rn(w.y);
-          wq[(size_t)(col + 2) * 64] = __float2bfloat16_rn(w.z);
-          wq[(size_t)(col + 3) * 64] = __float2bfloat16_rn(w.w);
+          wrow[i4 ^ (rloc & 7)] = w;
+          qrow[(4 * i4) * 64] = __float2bfloat16_rn(w.x);
+          qrow[(4 * i4 + 1) * 64] = __float2bfloat16_rn(w.y);
+          qrow[(4 * i4 + 2) * 64] = __float2bfloat16_rn(w.z);
+          qrow[(4 * i4 + 3) * 64] = __float2bfloat16_rn(w.w);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        group_barrier(1 + grp, 128);
+        if (leader) {
+          bulk_s2g(wn + (size_t)b * 4096, base_addr + L.off_w + s * DW1_WBLOCK, DW1_WBLOCK);
+          bulk_s2g(wq + (size_t)b * 2048, base_addr + L.off_q + grp * DW1_QSTAGE, 4096);
+          bulk_s2g(wq + (size_t)H * 64 + (size_t)b * 2048, base_addr + L.off_q + grp * DW1_QSTAGE + 4096, 4096);
+          bulk_commit();
+          bulk_wait_read_all();                         // shared memory read out (a fraction of a microsecond): slot and staging are free
+          mbar_arrive(wempty(s));
         }
       }
+      if (failed) break;
       tc_fence_before();                 // this warp's reads of the buffer are done: hand it back
       __syncwarp();
       if (lane == 0) mbar_arrive(acc_empty(buf));
     }
+    if (leader) bulk_wait_all();
+  } else {
+    // ---- w_j producer: the tile's blocks are consecutive 16 KB runs of the current version ----
+    if (lane == 0) {
+      auto tile_src = [&](int t) {
+        const int r = tile_r(t), slab = (t / parts) % slabs, part = t % parts;
+        return a.pool + ((size_t)r * a.n_slots + mlp_cur_slot(a, r, j)) * a.slot_stride +
+               (((size_t)slab * (H >> 5) + ((part * Hn) >> 5)) << 12);
+      };
+      const int nb = Hn / 32;
+      long long n = 0;
+      for (int t = blockIdx.x; t < n_tiles && !failed; t += gridDim.x) {
+        const float* src = tile_src(t);
+        if (t + (int)gridDim.x < n_tiles) bulk_prefetch_l2(tile_src(t + gridDim.x), (uint32_t)nb * DW1_WBLOCK);
+        for (int b = 0; b < nb; ++b, ++n) {
+          const int s = (int)(n % NB);
+          if (!mbar_wait(wempty(s), (uint32_t)(((n / NB) & 1) ^ 1))) { failed = true; break; }
+          mbar_arrive_expect_tx(wfull(s), DW1_WBLOCK);
+          bulk_g2s(base_addr + L.off_w + s * DW1_WBLOCK, src + (size_t)b * 4096, DW1_WBLOCK, wfull(s));
+        }
+      }
+    }
+    __syncwarp();
   }
 
   tc_fence_before();

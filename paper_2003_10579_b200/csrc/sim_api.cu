@@ -125,19 +125,24 @@ sim_status check_delay(const sim_handle* h, const sim_delay& dl) {
   return SIM_OK;
 }
 
-__global__ void broadcast_params_kernel(const float* w0, float* dst, long long n_params, long long stride, int R) {
+// tiled_dH / H: for the MLP the first tiled_dH parameters (W1) are stored block-tiled inside the pool
+__global__ void broadcast_params_kernel(const float* w0, float* dst, long long n_params, long long stride, int R,
+                                        long long tiled_dH, int H) {
   const long long total = n_params * R;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
     const long long r = i / n_params, p = i % n_params;
-    dst[r * stride + p] = w0[p];
+    const long long q = p < tiled_dH ? w1_tiled_index(p / H, p % H, H) : p;
+    dst[r * stride + q] = w0[p];
   }
 }
 
-__global__ void gather_params_kernel(const float* pool, const uint8_t* cur_slot, float* out, long long n_params, long long slot_stride, int n_slots, int R) {
+__global__ void gather_params_kernel(const float* pool, const uint8_t* cur_slot, float* out, long long n_params, long long slot_stride,
+                                     int n_slots, int R, long long tiled_dH, int H) {
   const long long total = n_params * R;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
     const long long r = i / n_params, p = i % n_params;
-    out[i] = pool[(r * n_slots + cur_slot[r]) * slot_stride + p];
+    const long long q = p < tiled_dH ? w1_tiled_index(p / H, p % H, H) : p;
+    out[i] = pool[(r * n_slots + cur_slot[r]) * slot_stride + q];
   }
 }
 
@@ -360,7 +365,9 @@ sim_status sim_set_params(sim_handle* h, const float* w0) {
   if (h->n_params == 0) return SIM_OK;
   float* dst = h->uses_pool ? h->pool : h->w_state;
   const long long stride = h->uses_pool ? (long long)h->n_slots * h->slot_stride : h->n_params;
-  broadcast_params_kernel<<<1184, 256, 0, h->stream>>>(w0, dst, h->n_params, stride, h->R);
+  const bool mlp = h->prob.model == SIM_MLP2;
+  broadcast_params_kernel<<<1184, 256, 0, h->stream>>>(w0, dst, h->n_params, stride, h->R,
+                                                        mlp ? (long long)h->prob.d * h->prob.hidden : 0, mlp ? h->prob.hidden : 1);
   CUDA_TRY(h, cudaGetLastError());
   // the caller's buffer is read by enqueued work: finish it before returning
   CUDA_TRY(h, cudaStreamSynchronize(h->stream));
@@ -518,7 +525,9 @@ sim_status sim_get_params(const sim_handle* h, float* w) {
   if (st != SIM_OK) return st;
   if (h->n_params == 0) return SIM_OK;
   if (h->uses_pool) {
-    gather_params_kernel<<<1184, 256, 0, h->stream>>>(h->pool, h->cur_slot, w, h->n_params, h->slot_stride, h->n_slots, h->R);
+    gather_params_kernel<<<1184, 256, 0, h->stream>>>(h->pool, h->cur_slot, w, h->n_params, h->slot_stride, h->n_slots, h->R,
+                                                       h->prob.model == SIM_MLP2 ? (long long)h->prob.d * h->prob.hidden : 0,
+                                                       h->prob.model == SIM_MLP2 ? h->prob.hidden : 1);
     CUDA_TRY(h, cudaGetLastError());
   } else {
     CUDA_TRY(h, cudaMemcpyAsync(w, h->w_state, (size_t)h->R * h->n_params * sizeof(float), cudaMemcpyDeviceToDevice, h->stream));
