@@ -1,8 +1,8 @@
 // Two-layer relu MLP (d - H - C, softmax cross-entropy) under the simulated schedule.
 //
 // Parameters per version: [W1 (d x H), b1 (H), W2 (H x C row-major), b2 (C)], fp32, kept in a pool of
-// immutable versions per replica (W1 block-tiled inside the pool, see w1_tiled_index; row-major to callers), plus a bf16 shadow of W1 per version and a
-// bf16 copy of the data set.  The two products over d take bf16 operands and accumulate in fp32
+// immutable versions per replica (W1 block-tiled inside the pool, see w1_tiled_index; row-major to
+// callers), plus a bf16 shadow of W1 per version and a bf16 copy of the data set.  The two products over d take bf16 operands and accumulate in fp32
 // on the tensor cores:
 //     A1 = bf16(X_b) bf16(W1)          (forward,  [m x d] [d x H])
 //     dW1 = bf16(X_b)^T bf16(delta1)   (backward, [d x m] [m x H])
@@ -13,12 +13,12 @@
 //   forward   (mlp_tc_kernel.cuh) one CTA per (replica, contributor, 128-sample block): A1 = X_b W1 on
 //             tcgen05 with the accumulator in tensor memory, then h = relu(A1 + b1), logits, softmax,
 //             delta2, delta1 = (delta2 W2^T) . [h > 0]; writes h, delta2, bf16(delta1), partial db1, loss
-//   head      one CTA per (replica, contributor): dW2 = h^T delta2, db2; the replica's last CTA then
-//             updates b1, W2, b2 from the partials (fixed summation order) and records the loss
-//   dw1       (mlp_tc_kernel.cuh) one CTA per (replica, 128-row slab of W1): accumulates X^T delta1 over
-//             all K m samples of the update in tensor memory (tcgen05, MN-major operands) and applies
-//             W1 <- W1 - (eta/(K m)) dW1 in its epilogue (Eq. 2 / Eq. 3), writing the new version and
-//             its transposed bf16 shadow: dW1 never exists in memory
+//   head      one CTA per (replica, 32 hidden units): dW2 = h^T delta2, db2 and db1 summed over the K
+//             contributors in a fixed order, b1 / W2 / b2 updated in the same CTA, loss recorded
+//   dw1       (mlp_tc_kernel.cuh) persistent, tiles of 128 rows of W1 x up to 256 columns: accumulates
+//             X^T delta1 over all K m samples of the update in tensor memory (tcgen05, MN-major
+//             operands) and applies W1 <- W1 - (eta/(K m)) dW1 in its epilogue (Eq. 2 / Eq. 3), writing
+//             the new version and its transposed bf16 shadow: dW1 never exists in memory
 #pragma once
 #include <cuda_bf16.h>
 
@@ -35,10 +35,7 @@ struct MlpScratch {
   float* Hact = nullptr;           // [R][Kmax][m][H]          h
   float* D2 = nullptr;             // [R][Kmax][m][16]         delta2
   float* db1_part = nullptr;       // [R][Kmax][m/32][H]       column sums of delta1 per 32-row group
-  float* dW2_part = nullptr;       // [R][Kmax][H*C]
-  float* db2_part = nullptr;       // [R][Kmax][16]
   float* loss_part = nullptr;      // [R][Kmax][m/32]
-  int* done_cnt = nullptr;         // [R]                      contributors whose head partials are complete
   int* rows_tab = nullptr;         // [R][Kmax][m]             sample row of every minibatch draw of the current update
   int H = 0, C = 0, d = 0, m = 0, Kmax = 0, n_slots = 0, R = 0;
   long long n = 0;
@@ -114,89 +111,102 @@ __global__ void mlp_rows_kernel(MlpArgs g) {
   }
 }
 
-// ---- b1, W2, b2 update and the loss record -------------------------------------------------------
-// (run by the last head CTA of a replica to finish: fixed summation order over contributors)
-__device__ void mlp_small_update(const MlpArgs& g, int r, int tid, int nthreads) {
+// ---- dW2 = h^T delta2, db2, db1 summed over the update's K contributors; b1, W2, b2 update; loss record ----
+// One CTA per (replica, 32 hidden columns): the K*m sample rows of the update are dealt to the eight warps
+// in chunks of 32 rows; a lane owns one column, holds the chunk's 32 activations in registers (32 loads
+// in flight) and reads the rows' delta2 from a per-warp shared-memory copy.  The eight warps' sums are
+// added in warp order, then the CTA applies Eq. 2 / Eq. 3 to its 32 rows of W2 and 32 entries of b1; the
+// CTA of columns 0..31 also owns b2 and the loss record.  Every sum has a fixed order.
+constexpr int MLP_HEAD_THREADS = 256;
+__global__ void __launch_bounds__(MLP_HEAD_THREADS, 3) mlp_head_kernel(MlpArgs g) {
   const NumericArgs& a = g.na;
   const MlpScratch& sc = g.sc;
+  const int H = sc.H, C = sc.C, m = sc.m, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int ncb = H / 32, cb = blockIdx.x % ncb, r = blockIdx.x / ncb;
   const long long j = g.j;
   const int K = (int)a.K_used[(size_t)r * a.cap + j];
-  const int H = sc.H, C = sc.C, m = sc.m, halves = m / 32;   // partial sums per 32-row group
+  const size_t row_base = (size_t)r * sc.Kmax * m;          // contributors l < K are consecutive blocks of m rows
+  const int n_chunks = K * m / 32;
+  __shared__ __align__(16) float d2_s[8][32][16];             // per warp: delta2 of the chunk's rows; later the warps' sums
+  float accw[16], accb = 0.f;
+#pragma unroll
+  for (int c = 0; c < 16; ++c) accw[c] = 0.f;
+  for (int ch = warp; ch < n_chunks; ch += 8) {
+    const size_t row0 = row_base + (size_t)ch * 32;
+    float hv[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) hv[i] = sc.Hact[(row0 + i) * H + cb * 32 + lane];
+    float4 dl[4];
+#pragma unroll
+    for (int c4 = 0; c4 < 4; ++c4) dl[c4] = reinterpret_cast<const float4*>(sc.D2 + (row0 + lane) * 16)[c4];
+    __syncwarp();
+#pragma unroll
+    for (int c4 = 0; c4 < 4; ++c4) reinterpret_cast<float4*>(&d2_s[warp][lane][0])[c4] = dl[c4];
+    __syncwarp();
+    if (cb == 0 && lane < 16) {                               // db2: lane c sums class c over the chunk's rows
+#pragma unroll 8
+      for (int i = 0; i < 32; ++i) accb += d2_s[warp][i][lane];
+    }
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+#pragma unroll
+      for (int c4 = 0; c4 < 4; ++c4) {
+        const float4 dv = reinterpret_cast<const float4*>(&d2_s[warp][i][0])[c4];
+        accw[4 * c4] = fmaf(hv[i], dv.x, accw[4 * c4]); accw[4 * c4 + 1] = fmaf(hv[i], dv.y, accw[4 * c4 + 1]);
+        accw[4 * c4 + 2] = fmaf(hv[i], dv.z, accw[4 * c4 + 2]); accw[4 * c4 + 3] = fmaf(hv[i], dv.w, accw[4 * c4 + 3]);
+      }
+    }
+  }
+  __syncwarp();
+#pragma unroll
+  for (int c4 = 0; c4 < 4; ++c4)
+    reinterpret_cast<float4*>(&d2_s[warp][lane][0])[c4] = make_float4(accw[4 * c4], accw[4 * c4 + 1], accw[4 * c4 + 2], accw[4 * c4 + 3]);
+  __shared__ float b2_s[8][16];
+  if (cb == 0 && lane < 16) b2_s[warp][lane] = accb;
+  __syncthreads();
+
   const long long dH = (long long)sc.d * H;
   const int cur = mlp_cur_slot(a, r, j), fresh = mlp_fresh_slot(a, r, j);
   const float scale = (float)((double)a.eta / ((double)K * (double)m));
-  const float* wc = a.pool + ((size_t)r * a.n_slots + cur) * a.slot_stride + dH;
+  const float* wc = a.pool + ((size_t)r * a.n_slots + cur) * a.slot_stride + dH;      // [b1 | W2 | b2] of w_j
   float* wn = a.pool + ((size_t)r * a.n_slots + fresh) * a.slot_stride + dH;
-  const int tail = H + H * C + C;
-  for (int p = tid; p < tail; p += nthreads) {
+  // W2 rows cb*32 .. cb*32+31: 32 x C consecutive parameters
+  for (int e = tid; e < 32 * C; e += MLP_HEAD_THREADS) {
+    const int col = e / C, c = e % C;
     float gsum = 0.f;
-    for (int l = 0; l < K; ++l) {
-      const size_t task = (size_t)r * sc.Kmax + l;
-      if (p < H) { for (int hf = 0; hf < halves; ++hf) gsum += sc.db1_part[(task * halves + hf) * H + p]; }
-      else if (p < H + H * C) gsum += sc.dW2_part[task * H * C + (p - H)];
-      else gsum += sc.db2_part[task * 16 + (p - H - H * C)];
-    }
+#pragma unroll
+    for (int w = 0; w < 8; ++w) gsum += d2_s[w][col][c];
+    const size_t p = (size_t)H + (size_t)(cb * 32) * C + e;
     wn[p] = fmaf(-scale, gsum, wc[p]);
   }
-  if (tid == 0) {
-    float ls = 0.f;
-    for (int l = 0; l < K; ++l)
-      for (int hf = 0; hf < halves; ++hf) ls += sc.loss_part[((size_t)r * sc.Kmax + l) * halves + hf];
-    a.loss[(size_t)r * a.cap + j] = ls / ((float)K * (float)m);
-    a.dist2[(size_t)r * a.cap + j] = 0.f;
+  if (tid < 32) {                                             // b1: partial column sums of delta1 written by the forward kernel
+    const int col = cb * 32 + tid, parts = m / 32;
+    float gsum = 0.f;
+    for (int q = 0; q < K * parts; ++q) gsum += sc.db1_part[((size_t)r * sc.Kmax * parts + q) * H + col];
+    wn[col] = fmaf(-scale, gsum, wc[col]);
   }
-}
-
-// ---- dW2 = h^T delta2, db2 (per contributor) --------------------------------------------------
-__global__ void __launch_bounds__(512) mlp_head_kernel(MlpArgs g) {
-  const NumericArgs& a = g.na;
-  const MlpScratch& sc = g.sc;
-  const int l = blockIdx.x % sc.Kmax, r = blockIdx.x / sc.Kmax;
-  const int K = (int)a.K_used[(size_t)r * a.cap + g.j];
-  if (l >= K) return;
-  const int H = sc.H, C = sc.C, m = sc.m, tid = threadIdx.x;
-  const size_t task = (size_t)r * sc.Kmax + l;
-  extern __shared__ __align__(128) unsigned char smem[];
-  float* d2_s = reinterpret_cast<float*>(smem);   // [m][16]
-  for (int i = tid; i < m * 16; i += blockDim.x) d2_s[i] = sc.D2[task * m * 16 + i];
-  __syncthreads();
-  if (tid < H) {
-    float accw[16];
+  if (cb == 0 && warp == 1) {
+    if (lane < C) {
+      float gsum = 0.f;
 #pragma unroll
-    for (int c = 0; c < 16; ++c) accw[c] = 0.f;
-    for (int row = 0; row < m; ++row) {
-      const float hv = sc.Hact[(task * m + row) * H + tid];
-#pragma unroll
-      for (int c4 = 0; c4 < 4; ++c4) {
-        const float4 dl = reinterpret_cast<const float4*>(d2_s + row * 16)[c4];
-        accw[4 * c4] = fmaf(hv, dl.x, accw[4 * c4]); accw[4 * c4 + 1] = fmaf(hv, dl.y, accw[4 * c4 + 1]);
-        accw[4 * c4 + 2] = fmaf(hv, dl.z, accw[4 * c4 + 2]); accw[4 * c4 + 3] = fmaf(hv, dl.w, accw[4 * c4 + 3]);
-      }
+      for (int w = 0; w < 8; ++w) gsum += b2_s[w][lane];
+      const size_t p = (size_t)H + (size_t)H * C + lane;
+      wn[p] = fmaf(-scale, gsum, wc[p]);
     }
-    for (int c = 0; c < C; ++c) sc.dW2_part[task * H * C + (size_t)tid * C + c] = accw[c];
-  }
-  if (tid < 16) {
-    float s = 0.f;
-    for (int row = 0; row < m; ++row) s += d2_s[row * 16 + tid];
-    sc.db2_part[task * 16 + tid] = s;
-  }
-  // the last of the replica's K contributor CTAs to get here applies the b1 / W2 / b2 update
-  __shared__ int is_last;
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) is_last = atomicAdd(&sc.done_cnt[r], 1) == K - 1;
-  __syncthreads();
-  if (is_last) {
-    __threadfence();
-    mlp_small_update(g, r, tid, blockDim.x);
-    if (tid == 0) sc.done_cnt[r] = 0;
+    if (lane == 31) {
+      const int parts = m / 32;
+      float ls = 0.f;
+      for (int q = 0; q < K * parts; ++q) ls += sc.loss_part[(size_t)r * sc.Kmax * parts + q];
+      a.loss[(size_t)r * a.cap + j] = ls / ((float)K * (float)m);
+      a.dist2[(size_t)r * a.cap + j] = 0.f;
+    }
   }
 }
 
 // ---- host side -----------------------------------------------------------------------------------
 inline void mlp_scratch_free(MlpScratch& s) {
-  cudaFree(s.done_cnt); cudaFree(s.rows_tab); cudaFree(s.Xq); cudaFree(s.W1qT); cudaFree(s.D1q); cudaFree(s.Hact); cudaFree(s.D2);
-  cudaFree(s.db1_part); cudaFree(s.dW2_part); cudaFree(s.db2_part); cudaFree(s.loss_part);
+  cudaFree(s.rows_tab); cudaFree(s.Xq); cudaFree(s.W1qT); cudaFree(s.D1q); cudaFree(s.Hact); cudaFree(s.D2);
+  cudaFree(s.db1_part); cudaFree(s.loss_part);
   s = MlpScratch{};
 }
 
@@ -214,11 +224,8 @@ inline cudaError_t mlp_scratch_alloc(MlpScratch& s, const float* X, long long n,
   MLP_ALLOC(s.Hact, tasks * m * H)
   MLP_ALLOC(s.D2, tasks * m * 16)
   MLP_ALLOC(s.db1_part, tasks * (m / 32) * H)
-  MLP_ALLOC(s.dW2_part, tasks * H * C)
-  MLP_ALLOC(s.db2_part, tasks * 16)
   MLP_ALLOC(s.loss_part, tasks * (m / 32))
   MLP_ALLOC(s.rows_tab, tasks * m)
-  MLP_ALLOC(s.done_cnt, (size_t)R)
 #undef MLP_ALLOC
   to_bf16_kernel<<<1184, 256, 0, stream>>>(X, s.Xq, (long long)n * d);
   return cudaGetLastError();

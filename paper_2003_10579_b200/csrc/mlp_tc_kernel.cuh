@@ -680,7 +680,7 @@ inline cudaError_t run_mlp(NumericArgs& a, MlpScratch& s, MlpMaps& maps, int P, 
     g.j = a.j0 + u;
     mlp_rows_kernel<<<a.R * s.Kmax, 128, 0, stream>>>(g);
     mlp_forward_tc_kernel<<<a.R * s.Kmax * mtiles, TC_THREADS, L.total, stream>>>(maps.tmX, maps.tmW, g);
-    mlp_head_kernel<<<a.R * s.Kmax, 512, (size_t)s.m * 16 * 4, stream>>>(g);
+    mlp_head_kernel<<<a.R * (s.H / 32), MLP_HEAD_THREADS, 0, stream>>>(g);
     mlp_dw1_tc_kernel<<<dw1_grid, DW1_THREADS, LD.total, stream>>>(maps.tmD, g);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
