@@ -399,9 +399,6 @@ __device__ __forceinline__ void bulk_s2g(void* dst, uint32_t src, uint32_t bytes
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes) {
-  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
-}
 __device__ __forceinline__ void group_barrier(int id, int threads) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory"); }
 
 __global__ void __launch_bounds__(DW1_THREADS, 1)
@@ -603,7 +600,6 @@ mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
       long long n = 0;
       for (int t = blockIdx.x; t < n_tiles && !failed; t += gridDim.x) {
         const float* src = tile_src(t);
-        if (t + (int)gridDim.x < n_tiles) bulk_prefetch_l2(tile_src(t + gridDim.x), (uint32_t)nb * DW1_WBLOCK);
         for (int b = 0; b < nb; ++b, ++n) {
           const int s = (int)(n % NB);
           if (!mbar_wait(wempty(s), (uint32_t)(((n / NB) & 1) ^ 1))) { failed = true; break; }
