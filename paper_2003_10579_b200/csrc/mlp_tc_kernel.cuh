@@ -5,10 +5,10 @@
 //   warp 0   B producer: TMA tensor loads of the W1 tile from the transposed, k-block-tiled bf16 shadow
 //            (K-major B operand, 128-byte swizzle; a stage's [H x 64] tile is one contiguous block of the
 //            shadow, fetched as one or two boxes)
-//   warps 2-5  A producer during the main loop: the 128 gathered sample rows of a stage are 1024
+//   warps 2-5  A producer during the main loop: the 128 gathered sample rows of a k-block are 1024
 //            16-byte pieces, copied with cp.async into the same 128-byte-swizzle pattern (one-row
 //            TMA boxes of 128 B were limited by the TMA instruction rate), made visible to the
-//            tensor core's asynchronous proxy with a proxy fence before the stage is signalled
+//            tensor core's asynchronous proxy with a proxy fence before the slot is signalled
 //   warp 1   allocates tensor memory; one elected lane issues tcgen05.mma (M=128, N<=256, K=16)
 //            and commits stage-free / accumulator-ready mbarriers
 //   warps 2-5  epilogue: tcgen05.ld gives each thread one sample's full row of A1, so bias, relu,
@@ -33,7 +33,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
-__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_alloc(uint32_t smem_dst, uint32_t ncols) {
@@ -76,20 +75,26 @@ __device__ __forceinline__ uint32_t tc_idesc(int n, int a_mn_major, int b_mn_maj
          ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
+constexpr int FWD_LAG = 2;    // k-blocks of A in flight per producer thread before the oldest is signalled
 struct TcLayout {   // shared-memory plan of the forward kernel (offsets from a 1024-byte aligned base)
-  int stages, stage_bytes, off_w2, off_b1, off_b2, off_rows, off_labels, off_bars, off_tmem, total;
+  int sa, sb, b_bytes, off_b, off_w2, off_b1, off_b2, off_rows, off_labels, off_bars, off_tmem, total;
 };
+// The operands have rings of their own: A (128 samples x 64 k, 16 KB) in `sa` slots; B in `sb` slots of
+// [n_inst x 64 k], n_inst = H (H <= 256) or H/2 - half a k-block of W1 per slot, so that several loads of
+// 32 KB are in flight instead of one of 64 KB.
 inline __host__ __device__ TcLayout tc_forward_layout(int H) {
   TcLayout L;
-  L.stage_bytes = TC_A_BYTES + H * 128;
-  L.stages = H <= 256 ? 4 : 2;
-  L.off_w2 = L.stages * L.stage_bytes;
+  L.b_bytes = (H > 256 ? H / 2 : H) * 128;
+  L.sa = 4;
+  L.sb = 3;
+  L.off_b = L.sa * TC_A_BYTES;
+  L.off_w2 = L.off_b + L.sb * L.b_bytes;
   L.off_b1 = L.off_w2 + H * 16 * 4;
   L.off_b2 = L.off_b1 + H * 4;
   L.off_rows = L.off_b2 + 64;
   L.off_labels = L.off_rows + 128 * 4;
   L.off_bars = L.off_labels + 128 * 4;
-  L.off_tmem = L.off_bars + 8 * (2 * L.stages + 1);
+  L.off_tmem = L.off_bars + 8 * (2 * L.sa + 2 * L.sb + 1);
   L.total = L.off_tmem + 16 + 1024;   // slack for the manual 1024-byte alignment
   return L;
 }
@@ -124,21 +129,24 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
   const uint32_t base_addr = (raw_addr + 1023u) & ~1023u;
   unsigned char* base = smem_raw + (base_addr - raw_addr);
   const TcLayout L = tc_forward_layout(H);
-  const int S = L.stages;
+  const int SA = L.sa, SB = L.sb;
   float* W2_s = reinterpret_cast<float*>(base + L.off_w2);
   float* b1_s = reinterpret_cast<float*>(base + L.off_b1);
   float* b2_s = reinterpret_cast<float*>(base + L.off_b2);
   int* rows_s = reinterpret_cast<int*>(base + L.off_rows);
   int* label_s = reinterpret_cast<int*>(base + L.off_labels);
-  const uint32_t bars = base_addr + L.off_bars;            // full[S] | empty[S] | acc_ready
+  const uint32_t bars = base_addr + L.off_bars;            // afull[SA] | aempty[SA] | bfull[SB] | bempty[SB] | acc_ready
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base + L.off_tmem);
-  auto full_bar = [&](int s) { return bars + 8u * s; };
-  auto empty_bar = [&](int s) { return bars + 8u * (S + s); };
-  const uint32_t acc_bar = bars + 8u * (2 * S);
+  auto afull = [&](int s) { return bars + 8u * s; };
+  auto aempty = [&](int s) { return bars + 8u * (SA + s); };
+  auto bfull = [&](int s) { return bars + 8u * (2 * SA + s); };
+  auto bempty = [&](int s) { return bars + 8u * (2 * SA + SB + s); };
+  const uint32_t acc_bar = bars + 8u * (2 * SA + 2 * SB);
 
   if (tid == 0) {
-    // a stage is full after the TMA bytes of B (one arrival with expect_tx) and the 128 A-producer threads
-    for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1 + 128); mbar_init(empty_bar(s), 1); }
+    // an A slot is full after its 128 producer threads arrived, a B slot after the TMA bytes (one arrival with expect_tx)
+    for (int s = 0; s < SA; ++s) { mbar_init(afull(s), 128); mbar_init(aempty(s), 1); }
+    for (int s = 0; s < SB; ++s) { mbar_init(bfull(s), 1); mbar_init(bempty(s), 1); }
     mbar_init(acc_bar, 1);
     mbar_fence_init();
   }
@@ -171,37 +179,39 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
     // ---- B producer ----
     const long long w_blk0 = ((long long)r * sc.n_slots + snap) * (d / TC_BK);     // first k-block of this W1^T shadow
     if (lane == 0) {
-      for (int kc = 0; kc < nk; ++kc) {
-        const int s = kc % S;
-        if (!mbar_wait(empty_bar(s), (uint32_t)(((kc / S) & 1) ^ 1))) { failed = true; break; }
-        const uint32_t Bs = base_addr + (uint32_t)s * L.stage_bytes + TC_A_BYTES;
-        mbar_arrive_expect_tx(full_bar(s), (uint32_t)(H * 128));
-        for (int hf = 0; hf < n_halves; ++hf)
-          tma_load_2d(Bs + (uint32_t)hf * n_inst * 128, &tmW, 0, (int)((w_blk0 + kc) * H + hf * n_inst), full_bar(s));
+      for (int n = 0; n < nk * n_halves; ++n) {
+        const int s = n % SB, kc = n / n_halves, hf = n % n_halves;
+        if (!mbar_wait(bempty(s), (uint32_t)(((n / SB) & 1) ^ 1))) { failed = true; break; }
+        mbar_arrive_expect_tx(bfull(s), (uint32_t)L.b_bytes);
+        tma_load_2d(base_addr + L.off_b + (uint32_t)s * L.b_bytes, &tmW, 0, (int)((w_blk0 + kc) * H + hf * n_inst), bfull(s));
       }
     }
     __syncwarp();
   } else if (warp == 1) {
     // ---- MMA issuer ----
     const uint32_t idesc = tc_idesc(n_inst, 0, 0);
-    for (int kc = 0; kc < nk; ++kc) {
-      const int s = kc % S;
-      if (!mbar_wait(full_bar(s), (uint32_t)((kc / S) & 1))) { failed = true; break; }
-      tc_fence_after();
-      if (lane == 0) {
-        const uint32_t As = base_addr + (uint32_t)s * L.stage_bytes, Bs = As + TC_A_BYTES;
+    for (int kc = 0; kc < nk && !failed; ++kc) {
+      const int sa = kc % SA;
+      if (!mbar_wait(afull(sa), (uint32_t)((kc / SA) & 1))) { failed = true; break; }
+      const uint32_t As = base_addr + (uint32_t)sa * TC_A_BYTES;
+      for (int hf = 0; hf < n_halves; ++hf) {
+        const int n = kc * n_halves + hf, s = n % SB;
+        if (!mbar_wait(bfull(s), (uint32_t)((n / SB) & 1))) { failed = true; break; }
+        tc_fence_after();
+        if (lane == 0) {
+          const uint32_t Bs = base_addr + L.off_b + (uint32_t)s * L.b_bytes;
 #pragma unroll
-        for (int k16 = 0; k16 < TC_BK / 16; ++k16) {
-          const uint64_t ad = tc_desc_kmajor(As + k16 * 32);
-          for (int hf = 0; hf < n_halves; ++hf) {
-            const uint64_t bd = tc_desc_kmajor(Bs + (uint32_t)hf * n_inst * 128 + k16 * 32);
-            tc_mma_bf16(tmem_base + (uint32_t)hf * n_inst, ad, bd, idesc, (kc > 0 || k16 > 0) ? 1u : 0u);
+          for (int k16 = 0; k16 < TC_BK / 16; ++k16)
+            tc_mma_bf16(tmem_base + (uint32_t)hf * n_inst, tc_desc_kmajor(As + k16 * 32), tc_desc_kmajor(Bs + k16 * 32), idesc,
+                        (kc > 0 || k16 > 0) ? 1u : 0u);
+          tc_commit(bempty(s));                     // the slot may be refilled once these MMAs have read it
+          if (hf == n_halves - 1) {
+            tc_commit(aempty(sa));
+            if (kc == nk - 1) tc_commit(acc_bar);   // accumulator complete
           }
         }
-        tc_commit(empty_bar(s));                    // the stage may be refilled once these MMAs have read it
-        if (kc == nk - 1) tc_commit(acc_bar);       // accumulator complete
+        __syncwarp();
       }
-      __syncwarp();
     }
   } else {
     // ---- epilogue: thread = one sample row ----
@@ -209,26 +219,28 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
     const int row = 32 * q + lane;
     const size_t grow = task * m + (size_t)mt * 128 + row;
     const int part = mt * 4 + q, parts = mtiles * 4;
-    // ---- A producer: thread t copies 16-byte piece (t & 7) of rows (t >> 3) + 16 i, i < 8 ----
+    // ---- A producer: thread t copies 16-byte piece (t & 7) of rows (t >> 3) + 16 i, i < 8.  A k-block is
+    //      signalled FWD_LAG k-blocks after it was issued; the ring is deeper than that (SA > FWD_LAG + 1), so
+    //      the signal never waits for a slot whose release depends on the k-block just before the signalled one.
     {
       const int t = tid - 64, ch = t & 7, row0 = t >> 3;
-      auto signal = [&](int kc2) {          // pieces of stage kc2 have landed: publish to the async proxy
+      auto signal = [&](int kc2) {          // pieces of k-block kc2 have landed: publish to the async proxy
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        mbar_arrive(full_bar(kc2 % S));
+        mbar_arrive(afull(kc2 % SA));
       };
       int signalled = 0;
       for (int kc = 0; kc < nk && !failed; ++kc) {
-        const int s = kc % S;
-        if (!mbar_wait(empty_bar(s), (uint32_t)(((kc / S) & 1) ^ 1))) { failed = true; break; }
-        const uint32_t As = base_addr + (uint32_t)s * L.stage_bytes;
+        const int s = kc % SA;
+        if (!mbar_wait(aempty(s), (uint32_t)(((kc / SA) & 1) ^ 1))) { failed = true; break; }
+        const uint32_t As = base_addr + (uint32_t)s * TC_A_BYTES;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const int rw = row0 + 16 * i;
           cp_async16(As + rw * 128 + ((ch ^ (rw & 7)) << 4), sc.Xq + (size_t)rows_s[rw] * d + (size_t)kc * TC_BK + ch * 8);
         }
         cp_async_commit();
-        if (kc >= S - 1) {                  // the group issued S-1 iterations ago is complete
-          if (S == 2) cp_async_wait<1>(); else cp_async_wait<3>();
+        if (kc >= FWD_LAG) {
+          cp_async_wait<FWD_LAG>();
           signal(signalled++);
         }
       }
@@ -433,7 +445,7 @@ mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
   auto wempty = [&](int s) { return bars + 8u * (2 * S + 4 + NB + s); };
 
   if (tid == 0) {
-    for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1 + 128); mbar_init(empty_bar(s), 1); }
+    for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1 + 128); mbar_init(empty_bar(s), 1); }    // B's expect_tx arrival + A's 128 producer threads
     for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 8); }
     for (int s = 0; s < NB; ++s) { mbar_init(wfull(s), 1); mbar_init(wempty(s), 1); }
     fail_s[0] = 0; fail_s[1] = 0;
@@ -496,8 +508,11 @@ mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
       }
     }
   } else if (warp < 6) {
-    // ---- A producers: thread p copies 16-byte piece (p & 15) of sample rows (p >> 4) + 8 i, i < 8 ----
+    // ---- A producers: thread p copies 16-byte piece (p & 15) of sample rows (p >> 4) + 8 i, i < 8.  A stage is
+    //      signalled `lag` stages after it was issued, lag = S - 2: the signal then never waits for a slot
+    //      whose release depends on the stage just before the signalled one.
     const int p = tid - 64, piece = p & 15, k0 = p >> 4;
+    const int lag = S > 2 ? S - 2 : 1;
     long long it = 0, signalled = 0;
     auto signal = [&](long long which) {
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -520,8 +535,8 @@ mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
                      sc.Xq + (size_t)rid[i] * d + (size_t)slab * 128 + piece * 8);
         }
         cp_async_commit();
-        if (it >= S - 1) {              // the group issued S-1 stages ago has landed
-          if (S == 2) cp_async_wait<1>(); else if (S == 3) cp_async_wait<2>(); else cp_async_wait<3>();
+        if (it >= lag) {                // the group issued `lag` stages ago has landed
+          if (lag == 1) cp_async_wait<1>(); else cp_async_wait<2>();
           signal(signalled++);
         }
       }
