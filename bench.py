@@ -121,6 +121,38 @@ def run_reference(args, wl):
     }))
 
 
+def run_profile_case(args, wl):
+    """One small run of another workload (first of its (variant, K) runs), for profiler captures."""
+    import torch
+    from paper_2003_10579_b200.binding import Simulation
+    wl = wl.scaled(n=args.profile_n)
+    data = wl.make_data()
+    dev = {"model": data["model"], "X": torch.from_numpy(data["X"]).cuda(), "y": torch.from_numpy(data["y"]).cuda(),
+           "n_classes": data["n_classes"], "hidden": data["hidden"]}
+    variant, K = wl.runs[0]
+    R = args.profile_replicas or wl.replicas
+    sim = Simulation(dev, P=wl.P, K=K, variant=variant, delay_kind=wl.delay_kind, mu=wl.mu, shift=wl.shift, eta=wl.eta,
+                     m=wl.m, seed=wl.seed, n_replicas=R)
+    if wl.t_interval > 0:
+        sim.set_adasync(wl.K0, args.profile_interval or wl.t_interval)
+    w0 = wl.w0()
+    if np.any(w0):
+        sim.set_params(torch.from_numpy(w0).cuda())
+    J = args.profile_updates
+    sim.reserve(J)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    sim.run(J)
+    e1.record()
+    torch.cuda.synchronize()
+    tr = sim.trace()
+    print(json.dumps({"profile_case": args.profile_case, "workload": wl.name, "variant": variant, "K": K, "n": args.profile_n,
+                      "replicas": R, "updates": J, "device_ms": e0.elapsed_time(e1), "last_loss": float(tr["loss"][0, -1])}))
+    sim.close()
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -133,9 +165,18 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--stages", type=int, default=0)
+    ap.add_argument("--profile-case", type=int, default=0, choices=[0, 3, 4, 5],
+                    help="instead of the benchmark, run workload 3, 4 or 5 once at --profile-n samples for "
+                         "--profile-updates updates (a capture-sized case for ncu) and print its device time")
+    ap.add_argument("--profile-n", type=int, default=65536)
+    ap.add_argument("--profile-updates", type=int, default=3)
+    ap.add_argument("--profile-replicas", type=int, default=0)
+    ap.add_argument("--profile-interval", type=float, default=0.0, help="AdaSync interval of the profile case (default: the workload's)")
     args = ap.parse_args()
 
     from paper_2003_10579_b200 import inputs
+    if args.profile_case:
+        return run_profile_case(args, inputs.WORKLOADS[args.profile_case])
     wl = inputs.WORKLOADS[2]
     if args.impl == "reference":
         return run_reference(args, wl)
