@@ -2,19 +2,22 @@
 // memory.
 //
 // One CTA per (replica, contributor, 128-sample block):  A1[128 x H] = bf16(X_b)[128 x d] bf16(W1)[d x H]
-//   warp 0   B producer: TMA tensor loads of the W1 tile from the transposed, k-block-tiled bf16 shadow
-//            (K-major B operand, 128-byte swizzle; a stage's [H x 64] tile is one contiguous block of the
-//            shadow, fetched as one or two boxes)
+//   warp 0   B producer: TMA tensor loads of W1 from the transposed, k-block-tiled bf16 shadow (K-major B
+//            operand, 128-byte swizzle), half a k-block ([H/2 x 64], contiguous in the shadow) per ring
+//            slot; the first slots are requested before the block's opening barrier
 //   warps 2-5  A producer during the main loop: the 128 gathered sample rows of a k-block are 1024
 //            16-byte pieces, copied with cp.async into the same 128-byte-swizzle pattern (one-row
 //            TMA boxes of 128 B were limited by the TMA instruction rate), made visible to the
 //            tensor core's asynchronous proxy with a proxy fence before the slot is signalled
 //   warp 1   allocates tensor memory; one elected lane issues tcgen05.mma (M=128, N<=256, K=16)
-//            and commits stage-free / accumulator-ready mbarriers
-//   warps 2-5  epilogue: tcgen05.ld gives each thread one sample's full row of A1, so bias, relu,
-//            the 10-way head, softmax and delta2 need no cross-thread reduction; a second pass
-//            over tensor memory forms delta1 = (delta2 W2^T) . [A1 + b1 > 0], stores it in bf16
-//            and reduces its column sums (db1) with a warp transposition reduce
+//            and commits slot-free / accumulator-ready mbarriers
+//   warps 6-9  during the main loop: stage b1, W2 (padded to 16 classes) and b2 of the snapshot
+//   warps 2-9  epilogue: tcgen05.ld gives each thread one sample's row of A1 - warps 2-5 the first
+//            half of the hidden units, warps 6-9 the second - so bias, relu and the partial logits
+//            need no cross-thread reduction; the two partial logit vectors of a row meet in shared
+//            memory, both threads form softmax and delta2, and a second pass over tensor memory
+//            forms delta1 = (delta2 W2^T) . [A1 + b1 > 0] for the own half, stores it in bf16 and
+//            reduces its column sums (db1) with a warp transposition reduce
 // Every mbarrier wait is bounded; a wait that runs out sets the error word and the CTA drains.
 #pragma once
 #include <cuda.h>
@@ -26,13 +29,15 @@ namespace ssim {
 
 constexpr int TC_BK = 64;                       // k per stage: one 128-byte swizzle atom of bf16
 constexpr int TC_A_BYTES = 128 * 128;           // 128 rows x 128 B
-constexpr int TC_THREADS = 192;
+constexpr int TC_THREADS = 320;      // warp 0 B producer, warp 1 MMA, warps 2-5 A producers + epilogue, warps 6-9 epilogue helpers
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
+// named barrier `id` (1..15) over `threads` threads (a multiple of 32)
+__device__ __forceinline__ void group_barrier(int id, int threads) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_alloc(uint32_t smem_dst, uint32_t ncols) {
@@ -77,7 +82,7 @@ __device__ __forceinline__ uint32_t tc_idesc(int n, int a_mn_major, int b_mn_maj
 
 constexpr int FWD_LAG = 2;    // k-blocks of A in flight per producer thread before the oldest is signalled
 struct TcLayout {   // shared-memory plan of the forward kernel (offsets from a 1024-byte aligned base)
-  int sa, sb, b_bytes, off_b, off_w2, off_b1, off_b2, off_rows, off_labels, off_bars, off_tmem, total;
+  int sa, sb, b_bytes, off_b, off_w2, off_b1, off_b2, off_rows, off_labels, off_zx, off_bars, off_tmem, total;
 };
 // The operands have rings of their own: A (128 samples x 64 k, 16 KB) in `sa` slots; B in `sb` slots of
 // [n_inst x 64 k], n_inst = H (H <= 256) or H/2 - half a k-block of W1 per slot, so that several loads of
@@ -93,7 +98,8 @@ inline __host__ __device__ TcLayout tc_forward_layout(int H) {
   L.off_b2 = L.off_b1 + H * 4;
   L.off_rows = L.off_b2 + 64;
   L.off_labels = L.off_rows + 128 * 4;
-  L.off_bars = L.off_labels + 128 * 4;
+  L.off_zx = L.off_labels + 128 * 4;              // partial logits of the two column halves: [2][128][16]
+  L.off_bars = L.off_zx + 2 * 128 * 16 * 4;
   L.off_tmem = L.off_bars + 8 * (2 * L.sa + 2 * L.sb + 1);
   L.total = L.off_tmem + 16 + 1024;   // slack for the manual 1024-byte alignment
   return L;
@@ -135,6 +141,7 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
   float* b2_s = reinterpret_cast<float*>(base + L.off_b2);
   int* rows_s = reinterpret_cast<int*>(base + L.off_rows);
   int* label_s = reinterpret_cast<int*>(base + L.off_labels);
+  float* zx_s = reinterpret_cast<float*>(base + L.off_zx);
   const uint32_t bars = base_addr + L.off_bars;            // afull[SA] | aempty[SA] | bfull[SB] | bempty[SB] | acc_ready
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base + L.off_tmem);
   auto afull = [&](int s) { return bars + 8u * s; };
@@ -150,36 +157,33 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
     mbar_init(acc_bar, 1);
     mbar_fence_init();
   }
+  const int nk = d / TC_BK;
+  const long long w_blk0 = ((long long)r * sc.n_slots + snap) * (d / TC_BK);     // first k-block of this W1^T shadow
+  const int n_first = min(SB, nk * n_halves);       // B loads that need no free slot: issued before the block barrier
+  if (tid == 0) {
+    for (int n = 0; n < n_first; ++n) {
+      mbar_arrive_expect_tx(bfull(n), (uint32_t)L.b_bytes);
+      tma_load_2d(base_addr + L.off_b + (uint32_t)n * L.b_bytes, &tmW, 0, (int)((w_blk0 + n / n_halves) * H + (n % n_halves) * n_inst), bfull(n));
+    }
+  }
   if (warp == 1) tc_alloc(smem_addr(tmem_slot), tmem_cols);
-  {
-    const float* b1 = wsnap + dH;
-    const float* W2 = b1 + H;
-    const float* b2 = W2 + (size_t)H * C;
-    for (int i = tid; i < H * 16; i += TC_THREADS) {
-      const int col = i >> 4, c = i & 15;
-      W2_s[i] = c < C ? W2[(size_t)col * C + c] : 0.f;
-    }
-    for (int i = tid; i < H; i += TC_THREADS) b1_s[i] = b1[i];
-    if (tid < 16) b2_s[tid] = tid < C ? b2[tid] : 0.f;
-    if (tid < 128) {
-      uint32_t idx = draw_index(a.seed, rid, worker, seq, (uint32_t)(mt * 128 + tid), a.n);
-      if ((uint64_t)idx >= a.n) { atomicExch(a.err, ERR_BAD_INDEX); idx = 0; }
-      rows_s[tid] = (int)idx;
-      label_s[tid] = reinterpret_cast<const int*>(a.y)[idx];
-    }
+  if (tid >= 64 && tid < 192) {                     // the minibatch: sample rows and labels (the A producers need them first)
+    const int t = tid - 64;
+    uint32_t idx = draw_index(a.seed, rid, worker, seq, (uint32_t)(mt * 128 + t), a.n);
+    if ((uint64_t)idx >= a.n) { atomicExch(a.err, ERR_BAD_INDEX); idx = 0; }
+    rows_s[t] = (int)idx;
+    label_s[t] = reinterpret_cast<const int*>(a.y)[idx];
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const int nk = d / TC_BK;
   bool failed = false;
 
   if (warp == 0) {
     // ---- B producer ----
-    const long long w_blk0 = ((long long)r * sc.n_slots + snap) * (d / TC_BK);     // first k-block of this W1^T shadow
     if (lane == 0) {
-      for (int n = 0; n < nk * n_halves; ++n) {
+      for (int n = n_first; n < nk * n_halves; ++n) {
         const int s = n % SB, kc = n / n_halves, hf = n % n_halves;
         if (!mbar_wait(bempty(s), (uint32_t)(((n / SB) & 1) ^ 1))) { failed = true; break; }
         mbar_arrive_expect_tx(bfull(s), (uint32_t)L.b_bytes);
@@ -214,11 +218,26 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
       }
     }
   } else {
-    // ---- epilogue: thread = one sample row ----
+    // ---- warps 2-9: thread = one sample row and one half of the hidden units in the epilogue ----
     const int q = warp & 3;                         // the TMEM lane quarter this warp may read
+    const int ehalf = warp >= 6 ? 1 : 0;            // hidden units [ehalf * H/2, +H/2)
     const int row = 32 * q + lane;
     const size_t grow = task * m + (size_t)mt * 128 + row;
     const int part = mt * 4 + q, parts = mtiles * 4;
+    if (ehalf) {
+      // ---- helpers, during the main loop: b1, W2 (rows padded to 16 classes) and b2 of the snapshot ----
+      const int t = tid - 192;
+      const float* b1 = wsnap + dH;
+      const float* W2 = b1 + H;
+      const float* b2 = W2 + (size_t)H * C;
+#pragma unroll 8
+      for (int i = t; i < H * 16; i += 128) {
+        const int col = i >> 4, c = i & 15;
+        W2_s[i] = c < C ? W2[(size_t)col * C + c] : 0.f;
+      }
+      for (int i = t; i < H; i += 128) b1_s[i] = b1[i];
+      if (t < 16) b2_s[t] = t < C ? b2[t] : 0.f;
+    } else
     // ---- A producer: thread t copies 16-byte piece (t & 7) of rows (t >> 3) + 16 i, i < 8.  A k-block is
     //      signalled FWD_LAG k-blocks after it was issued; the ring is deeper than that (SA > FWD_LAG + 1), so
     //      the signal never waits for a slot whose release depends on the k-block just before the signalled one.
@@ -247,15 +266,17 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
       cp_async_wait<0>();
       if (!failed) while (signalled < nk) signal(signalled++);
     }
+    group_barrier(1, 256);                          // b1 / W2 / b2 are in shared memory (all eight warps, failed or not)
     if (!failed && !mbar_wait(acc_bar, 0)) failed = true;
     tc_fence_after();
+    const uint32_t trow = tmem_base + ((uint32_t)(32 * q) << 16);
+    const int ch0 = ehalf * (H / 64), ch1 = ch0 + H / 64;
+    float z[16];
+    uint32_t v[32];
     if (!failed) {
-      const uint32_t trow = tmem_base + ((uint32_t)(32 * q) << 16);
-      float z[16];
 #pragma unroll
-      for (int c = 0; c < 16; ++c) z[c] = b2_s[c];
-      uint32_t v[32];
-      for (int ch = 0; ch < H / 32; ++ch) {
+      for (int c = 0; c < 16; ++c) z[c] = 0.f;
+      for (int ch = ch0; ch < ch1; ++ch) {
         tc_ld32(trow + ch * 32, v);
         float4* hout = reinterpret_cast<float4*>(sc.Hact + grow * H + ch * 32);
 #pragma unroll
@@ -278,6 +299,15 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
           hout[i4] = make_float4(hv[0], hv[1], hv[2], hv[3]);
         }
       }
+#pragma unroll
+      for (int c4 = 0; c4 < 4; ++c4)
+        reinterpret_cast<float4*>(zx_s + (ehalf * 128 + row) * 16)[c4] = make_float4(z[4 * c4], z[4 * c4 + 1], z[4 * c4 + 2], z[4 * c4 + 3]);
+    }
+    group_barrier(1, 256);                          // both halves of every row's logits are published
+    if (!failed) {
+      // logits = b2 + half 0 + half 1, in this order in both threads of the row
+#pragma unroll
+      for (int c = 0; c < 16; ++c) z[c] = (b2_s[c] + zx_s[row * 16 + c]) + zx_s[(128 + row) * 16 + c];
       // softmax cross-entropy of this row; exponentials without the maximal class keep log(1+s)
       // and p_max - 1 = -s/(1+s) accurate for wide margins
       const int lab = label_s[row];
@@ -304,14 +334,16 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
         }
         d2[c] = dl;
       }
+      if (!ehalf) {
 #pragma unroll
-      for (int c4 = 0; c4 < 4; ++c4)
-        reinterpret_cast<float4*>(sc.D2 + grow * 16)[c4] = make_float4(d2[4 * c4], d2[4 * c4 + 1], d2[4 * c4 + 2], d2[4 * c4 + 3]);
-      float rowloss = warp_sum(log1pf(sexcl) + (zmax - zl));
-      if (lane == 0) sc.loss_part[task * parts + part] = rowloss;
+        for (int c4 = 0; c4 < 4; ++c4)
+          reinterpret_cast<float4*>(sc.D2 + grow * 16)[c4] = make_float4(d2[4 * c4], d2[4 * c4 + 1], d2[4 * c4 + 2], d2[4 * c4 + 3]);
+        float rowloss = warp_sum(log1pf(sexcl) + (zmax - zl));
+        if (lane == 0) sc.loss_part[task * parts + part] = rowloss;
+      }
 
-      // second pass: delta1, its bf16 copy and its column sums over this warp's 32 rows
-      for (int ch = 0; ch < H / 32; ++ch) {
+      // second pass: delta1, its bf16 copy and its column sums over this warp's 32 rows, own half of the units
+      for (int ch = ch0; ch < ch1; ++ch) {
         tc_ld32(trow + ch * 32, v);
         float dv[32];
 #pragma unroll
@@ -411,7 +443,6 @@ __device__ __forceinline__ void bulk_s2g(void* dst, uint32_t src, uint32_t bytes
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void group_barrier(int id, int threads) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory"); }
 
 __global__ void __launch_bounds__(DW1_THREADS, 1)
 mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
