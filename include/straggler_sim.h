@@ -30,7 +30,7 @@
 extern "C" {
 #endif
 
-#define SIM_MAX_P 32          /* workers per replica (one warp lane each in the arrival kernels) */
+#define SIM_MAX_P 128         /* workers per replica (a warp per replica in the arrival kernel: 1, 2 or 4 workers per lane) */
 #define SIM_MAX_CLASSES 16    /* softmax / MLP outputs */
 
 typedef struct sim_handle sim_handle;   /* opaque; owned by the library */
@@ -233,7 +233,7 @@ sim_status sim_sweep_host(const sim_problem* problem, int32_t P, int32_t n_runs,
  *   K_max = K, or P when t_interval > 0 (then K0 is the first K and K is ignored).
  * The per-replica worker state lives in one fixed array inside the library image
  * (SIM_NOALLOC_SCRATCH_BYTES of device memory on every GPU that loads the library, held until the
- * process exits), which bounds the problem: n_replicas <= SIM_NOALLOC_MAX_REPLICAS and
+ * process exits), which bounds the problem: P <= SIM_NOALLOC_MAX_P, n_replicas <= SIM_NOALLOC_MAX_REPLICAS and
  * n_replicas * P <= SIM_NOALLOC_MAX_REPLICA_WORKERS; larger requests return SIM_ERR_ARG and launch
  * nothing.  The first call on each device looks up the array's device address; make that first
  * call outside any stream capture.  All calls on a device share the array and each call clears
@@ -241,6 +241,7 @@ sim_status sim_sweep_host(const sim_problem* problem, int32_t P, int32_t n_runs,
  * threads) race: serialise them.  Work is enqueued on `cuda_stream`; the call does not wait for
  * it.  On failure sim_noalloc_last_error() describes the cause (per host thread).
  */
+#define SIM_NOALLOC_MAX_P 32   /* sim_schedule_noalloc: one warp lane per worker */
 #define SIM_NOALLOC_MAX_REPLICAS 4096
 #define SIM_NOALLOC_MAX_REPLICA_WORKERS 65536
 #define SIM_NOALLOC_SCRATCH_BYTES (1088 * 1024)

@@ -205,7 +205,7 @@ sim_status sim_schedule_noalloc(int32_t P, int32_t K, sim_variant variant, sim_d
                                 int64_t replica_base, int32_t n_replicas, int32_t K0, double t_interval,
                                 int64_t iters, double* t, uint16_t* K_used, uint16_t* worker,
                                 uint32_t* stale, uint32_t* seq, void* cuda_stream) {
-  if (P < 1 || P > SIM_MAX_P) return na_fail(SIM_ERR_ARG, "P must be in [1, SIM_MAX_P]");
+  if (P < 1 || P > SIM_NOALLOC_MAX_P) return na_fail(SIM_ERR_ARG, "P must be in [1, SIM_NOALLOC_MAX_P]");
   if ((int)variant < 0 || (int)variant > 3) return na_fail(SIM_ERR_ARG, "unknown variant");
   const bool growing = t_interval > 0.0;
   if (growing ? (K0 < 1 || K0 > P) : (K < 1 || K > P)) return na_fail(SIM_ERR_ARG, "K (or K0) must be in [1, P]");

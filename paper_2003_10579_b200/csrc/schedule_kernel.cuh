@@ -1,5 +1,5 @@
 // Arrival process of the four SGD variants of Section 2.2: one warp per replica, one lane per
-// worker (P <= 32).  The process depends on the delay stream only, never on parameter values,
+// worker for P <= 32, two or four workers per lane for P <= 64 / P <= 128.  The process depends on the delay stream only, never on parameter values,
 // so it runs ahead of the numeric kernels and leaves them a compact schedule:
 //   per update j: clock t_{j+1} (fp64), K_j, and for each contributor in arrival order its
 //   worker id, task sequence number, staleness j - tau and (asynchronous variants) the slot of
@@ -68,18 +68,31 @@ __device__ __forceinline__ bool before(double va, int ia, double vb, int ib) {
   return va < vb || (va == vb && ia < ib);
 }
 
-// number of workers that arrive strictly before (v, lane)
-__device__ __forceinline__ int arrival_rank(double v, int lane, int P) {
-  int rank = 0;
-  for (int o = 0; o < P; ++o) {
-    const double vo = __shfl_sync(0xFFFFFFFFu, v, o);
-    rank += before(vo, o, v, lane) ? 1 : 0;
+// Lane `lane` owns workers lane, lane + 32, ..., lane + 32 (I - 1): I = 1 for P <= 32, 2 for P <= 64,
+// 4 for P <= 128.  Everything below is unrolled over the I items, so I = 1 is the one-lane-per-worker code.
+
+// rank[i] = number of workers that arrive strictly before worker lane + 32 i
+template <int I>
+__device__ __forceinline__ void arrival_ranks(const double (&v)[I], int lane, int P, int (&rank)[I]) {
+#pragma unroll
+  for (int i = 0; i < I; ++i) rank[i] = 0;
+#pragma unroll
+  for (int ob = 0; ob < I; ++ob) {
+    for (int o = 0; o < 32 && ob * 32 + o < P; ++o) {
+      const double vo = __shfl_sync(0xFFFFFFFFu, v[ob], o);
+#pragma unroll
+      for (int i = 0; i < I; ++i) rank[i] += before(vo, ob * 32 + o, v[i], lane + 32 * i) ? 1 : 0;
+    }
   }
-  return rank;
 }
 
-__device__ __forceinline__ void warp_argmin(double v, int lane, double& bv, int& bi) {
-  bv = v; bi = lane;
+// value and worker id of the earliest (time, id) over all workers of the warp
+template <int I>
+__device__ __forceinline__ void warp_argmin(const double (&v)[I], int lane, double& bv, int& bi) {
+  bv = v[0]; bi = lane;
+#pragma unroll
+  for (int i = 1; i < I; ++i)
+    if (before(v[i], lane + 32 * i, bv, bi)) { bv = v[i]; bi = lane + 32 * i; }
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) {
     const double ov = __shfl_xor_sync(0xFFFFFFFFu, bv, off);
@@ -88,26 +101,81 @@ __device__ __forceinline__ void warp_argmin(double v, int lane, double& bv, int&
   }
 }
 
-__device__ __forceinline__ unsigned long long warp_or64(unsigned long long m) {
-  const uint32_t lo = __reduce_or_sync(0xFFFFFFFFu, (uint32_t)m);
-  const uint32_t hi = __reduce_or_sync(0xFFFFFFFFu, (uint32_t)(m >> 32));
-  return ((unsigned long long)hi << 32) | lo;
+// the value item `id >> 5` of lane `id & 31` holds
+template <int I>
+__device__ __forceinline__ int item_of_worker(const int (&x)[I], int id) {
+  int out = 0;
+#pragma unroll
+  for (int i = 0; i < I; ++i) {
+    const int t = __shfl_sync(0xFFFFFFFFu, x[i], id & 31);
+    if ((id >> 5) == i) out = t;
+  }
+  return out;
+}
+template <int I>
+__device__ __forceinline__ double item_of_worker(const double (&x)[I], int id) {
+  double out = 0.0;
+#pragma unroll
+  for (int i = 0; i < I; ++i) {
+    const double t = __shfl_sync(0xFFFFFFFFu, x[i], id & 31);
+    if ((id >> 5) == i) out = t;
+  }
+  return out;
 }
 
+// Set of version-pool slots (at most 32 I + 2 of them) as I + 1 words.
+template <int I>
+struct SlotSet {
+  uint32_t w[I + 1];
+  __device__ __forceinline__ void clear() {
+#pragma unroll
+    for (int k = 0; k <= I; ++k) w[k] = 0u;
+  }
+  __device__ __forceinline__ void add(int slot) {
+#pragma unroll
+    for (int k = 0; k <= I; ++k) if ((slot >> 5) == k) w[k] |= 1u << (slot & 31);
+  }
+  __device__ __forceinline__ void warp_union() {
+#pragma unroll
+    for (int k = 0; k <= I; ++k) w[k] = __reduce_or_sync(0xFFFFFFFFu, w[k]);
+  }
+  __device__ __forceinline__ void join(const SlotSet& o) {
+#pragma unroll
+    for (int k = 0; k <= I; ++k) w[k] |= o.w[k];
+  }
+  __device__ __forceinline__ int first_free() const {     // lowest slot not in the set, or 32 (I + 1)
+    int out = 32 * (I + 1);
+#pragma unroll
+    for (int k = I; k >= 0; --k) if (~w[k]) out = 32 * k + __ffs((int)~w[k]) - 1;
+    return out;
+  }
+};
+
+template <int I>
 __global__ void __launch_bounds__(128) schedule_kernel(ScheduleArgs a) {
   const int lane = threadIdx.x & 31;
   const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (r >= a.R) return;
   const int P = a.P;
-  const bool active = lane < P;
   const uint32_t rid = a.replica_base + (uint32_t)r;
   const bool async = a.variant == V_KASYNC || a.variant == V_KBATCHASYNC;
   const double INF = __longlong_as_double(0x7FF0000000000000ll);
 
-  uint32_t s = active ? a.s[r * P + lane] : 0u;
-  uint32_t tau = active ? a.tau[r * P + lane] : 0u;
-  double f = (active && async) ? a.f[r * P + lane] : INF;
-  int slot = (active && async) ? a.wslot[r * P + lane] : 0;
+  bool active[I];
+  uint32_t s[I], tau[I];
+  double f[I];
+  int slot[I];
+  bool fresh_start = true;
+#pragma unroll
+  for (int i = 0; i < I; ++i) {
+    const int id = lane + 32 * i;
+    active[i] = id < P;
+    s[i] = active[i] ? a.s[r * P + id] : 0u;
+    tau[i] = active[i] ? a.tau[r * P + id] : 0u;
+    f[i] = (active[i] && async) ? a.f[r * P + id] : INF;
+    slot[i] = (active[i] && async) ? a.wslot[r * P + id] : 0;
+    fresh_start = fresh_start && s[i] == 0u;
+  }
   int cur = async ? a.cur_slot[r] : 0;
   double clock = a.clock[r];
 
@@ -115,8 +183,10 @@ __global__ void __launch_bounds__(128) schedule_kernel(ScheduleArgs a) {
   const long long j_begin = j, j_end = a.adaptive ? a.target : a.j0 + a.iters;
   int K_now = a.adaptive ? a.K_cur[r] : 0, want = 0;
   long long q_last = a.adaptive ? a.q_last[r] : 0;
-  if (async && j == 0 && __all_sync(0xFFFFFFFFu, s == 0u)) {   // every worker fetches w_0 and starts its first minibatch at t = 0
-    if (active) { f = __dadd_rn(0.0, draw_delay(a.law, a.seed, rid, lane, s)); s += 1; tau = 0; slot = 0; }
+  if (async && j == 0 && __all_sync(0xFFFFFFFFu, fresh_start)) {   // every worker fetches w_0 and starts its first minibatch at t = 0
+#pragma unroll
+    for (int i = 0; i < I; ++i)
+      if (active[i]) { f[i] = __dadd_rn(0.0, draw_delay(a.law, a.seed, rid, lane + 32 * i, s[i])); s[i] += 1; tau[i] = 0; slot[i] = 0; }
     cur = 0;
   }
   if (async && lane == 0) a.begin_slot[r] = (uint8_t)cur;
@@ -144,64 +214,109 @@ __global__ void __launch_bounds__(128) schedule_kernel(ScheduleArgs a) {
     }
 
     if (a.variant == V_KSYNC) {
-      double x = INF;
-      if (active) { x = draw_delay(a.law, a.seed, rid, lane, s); s += 1; }
-      const int rank = arrival_rank(x, lane, P);
-      if (active && rank < K) { wk[rank] = (uint16_t)lane; sl[rank] = 0u; sq[rank] = s - 1u; }
-      const unsigned who = __ballot_sync(0xFFFFFFFFu, active && rank == K - 1);
-      const double T = __shfl_sync(0xFFFFFFFFu, x, __ffs(who) - 1);
+      double x[I];
+      int rank[I];
+#pragma unroll
+      for (int i = 0; i < I; ++i) {
+        x[i] = INF;
+        if (active[i]) { x[i] = draw_delay(a.law, a.seed, rid, lane + 32 * i, s[i]); s[i] += 1; }
+      }
+      arrival_ranks<I>(x, lane, P, rank);
+      double T = 0.0;
+#pragma unroll
+      for (int i = 0; i < I; ++i) {
+        if (active[i] && rank[i] < K) { wk[rank[i]] = (uint16_t)(lane + 32 * i); sl[rank[i]] = 0u; sq[rank[i]] = s[i] - 1u; }
+        const unsigned who = __ballot_sync(0xFFFFFFFFu, active[i] && rank[i] == K - 1);
+        const double Ti = __shfl_sync(0xFFFFFFFFu, x[i], who ? __ffs(who) - 1 : 0);
+        if (who) T = Ti;
+      }
       clock = __dadd_rn(clock, T);
     } else if (a.variant == V_KBATCHSYNC) {
-      double c = INF;
-      if (active) { c = draw_delay(a.law, a.seed, rid, lane, s); s += 1; }
+      double c[I];
+#pragma unroll
+      for (int i = 0; i < I; ++i) {
+        c[i] = INF;
+        if (active[i]) { c[i] = draw_delay(a.law, a.seed, rid, lane + 32 * i, s[i]); s[i] += 1; }
+      }
       double T = 0.0;
       for (int l = 0; l < K; ++l) {
         double bv; int bi;
-        warp_argmin(c, lane, bv, bi);
+        warp_argmin<I>(c, lane, bv, bi);
         T = bv;
-        if (lane == bi) {
-          wk[l] = (uint16_t)lane; sl[l] = 0u; sq[l] = s - 1u;
-          if (l + 1 < K) { c = __dadd_rn(c, draw_delay(a.law, a.seed, rid, lane, s)); s += 1; }
+#pragma unroll
+        for (int i = 0; i < I; ++i) {
+          if (bi == lane + 32 * i) {
+            wk[l] = (uint16_t)bi; sl[l] = 0u; sq[l] = s[i] - 1u;
+            if (l + 1 < K) { c[i] = __dadd_rn(c[i], draw_delay(a.law, a.seed, rid, bi, s[i])); s[i] += 1; }
+          }
         }
       }
       clock = __dadd_rn(clock, T);
     } else if (a.variant == V_KASYNC) {
-      const int rank = arrival_rank(f, lane, P);
-      const bool mine = active && rank < K;
-      if (mine) { wk[rank] = (uint16_t)lane; sl[rank] = (uint32_t)(j - (long long)tau); sq[rank] = s - 1u; ss[rank] = (uint8_t)slot; }
-      const unsigned who = __ballot_sync(0xFFFFFFFFu, active && rank == K - 1);
-      clock = __shfl_sync(0xFFFFFFFFu, f, __ffs(who) - 1);
+      int rank[I];
+      arrival_ranks<I>(f, lane, P, rank);
+      bool mine[I];
+      double t_new = 0.0;
+      SlotSet<I> used;
+      used.clear();
+#pragma unroll
+      for (int i = 0; i < I; ++i) {
+        mine[i] = active[i] && rank[i] < K;
+        if (mine[i]) {
+          wk[rank[i]] = (uint16_t)(lane + 32 * i); sl[rank[i]] = (uint32_t)(j - (long long)tau[i]); sq[rank[i]] = s[i] - 1u;
+          ss[rank[i]] = (uint8_t)slot[i];
+        }
+        const unsigned who = __ballot_sync(0xFFFFFFFFu, active[i] && rank[i] == K - 1);
+        const double ti = __shfl_sync(0xFFFFFFFFu, f[i], who ? __ffs(who) - 1 : 0);
+        if (who) t_new = ti;
+        if (active[i]) used.add(slot[i]);
+      }
+      clock = t_new;
       // w_{j+1} goes to a slot that no worker holds and that is not w_j
-      const unsigned long long used = warp_or64(active ? (1ull << slot) : 0ull) | (1ull << cur);
-      int fresh = __ffsll((long long)~used) - 1;
-      if (fresh < 0 || fresh >= a.n_slots) { if (lane == 0) atomicExch(a.err, ERR_NO_FREE_SLOT); fresh = 0; }
+      used.warp_union();
+      used.add(cur);
+      int fresh = used.first_free();
+      if (fresh >= a.n_slots) { if (lane == 0) atomicExch(a.err, ERR_NO_FREE_SLOT); fresh = 0; }
       if (lane == 0) a.new_slot[row] = (uint8_t)fresh;
-      if (mine) {
-        tau = (uint32_t)(j + 1); slot = fresh;
-        f = __dadd_rn(clock, draw_delay(a.law, a.seed, rid, lane, s)); s += 1;
+#pragma unroll
+      for (int i = 0; i < I; ++i) {
+        if (mine[i]) {
+          tau[i] = (uint32_t)(j + 1); slot[i] = fresh;
+          f[i] = __dadd_rn(clock, draw_delay(a.law, a.seed, rid, lane + 32 * i, s[i])); s[i] += 1;
+        }
       }
       cur = fresh;
     } else {  // V_KBATCHASYNC
-      unsigned long long read_now = 0ull;   // slots whose parameters this update's gradients read
+      SlotSet<I> read_now;                  // slots whose parameters this update's gradients read
+      read_now.clear();
       for (int l = 0; l < K; ++l) {
         double bv; int bi;
-        warp_argmin(f, lane, bv, bi);
-        const int bslot = __shfl_sync(0xFFFFFFFFu, slot, bi);
-        read_now |= 1ull << bslot;
+        warp_argmin<I>(f, lane, bv, bi);
+        const int bslot = item_of_worker<I>(slot, bi);
+        read_now.add(bslot);
         int fresh = cur;
         if (l + 1 == K) {
           clock = bv;
-          const unsigned long long used = warp_or64(active ? (1ull << slot) : 0ull) | (1ull << cur) | read_now;
-          fresh = __ffsll((long long)~used) - 1;
-          if (fresh < 0 || fresh >= a.n_slots) { if (lane == 0) atomicExch(a.err, ERR_NO_FREE_SLOT); fresh = 0; }
+          SlotSet<I> used;
+          used.clear();
+#pragma unroll
+          for (int i = 0; i < I; ++i) if (active[i]) used.add(slot[i]);
+          used.warp_union();
+          used.add(cur);
+          used.join(read_now);
+          fresh = used.first_free();
+          if (fresh >= a.n_slots) { if (lane == 0) atomicExch(a.err, ERR_NO_FREE_SLOT); fresh = 0; }
           if (lane == 0) a.new_slot[row] = (uint8_t)fresh;
         }
-        if (lane == bi) {
-          wk[l] = (uint16_t)lane; sl[l] = (uint32_t)(j - (long long)tau); sq[l] = s - 1u; ss[l] = (uint8_t)slot;
-          // the pusher fetches what the server holds after its push was counted
-          tau = (l + 1 == K) ? (uint32_t)(j + 1) : (uint32_t)j;
-          slot = fresh;
-          f = __dadd_rn(f, draw_delay(a.law, a.seed, rid, lane, s)); s += 1;
+#pragma unroll
+        for (int i = 0; i < I; ++i) {
+          if (bi == lane + 32 * i) {
+            wk[l] = (uint16_t)bi; sl[l] = (uint32_t)(j - (long long)tau[i]); sq[l] = s[i] - 1u; ss[l] = (uint8_t)slot[i];
+            // the pusher fetches what the server holds after its push was counted
+            tau[i] = (l + 1 == K) ? (uint32_t)(j + 1) : (uint32_t)j;
+            slot[i] = fresh;
+            f[i] = __dadd_rn(f[i], draw_delay(a.law, a.seed, rid, bi, s[i])); s[i] += 1;
+          }
         }
         if (l + 1 == K) cur = fresh;
       }
@@ -209,10 +324,14 @@ __global__ void __launch_bounds__(128) schedule_kernel(ScheduleArgs a) {
     if (lane == 0) { a.t[row] = clock; a.K_used[row] = (uint16_t)K; }
   }
 
-  if (active) {
-    a.s[r * P + lane] = s;
-    a.tau[r * P + lane] = tau;
-    if (async) { a.f[r * P + lane] = f; a.wslot[r * P + lane] = (uint8_t)slot; }
+#pragma unroll
+  for (int i = 0; i < I; ++i) {
+    const int id = lane + 32 * i;
+    if (active[i]) {
+      a.s[r * P + id] = s[i];
+      a.tau[r * P + id] = tau[i];
+      if (async) { a.f[r * P + id] = f[i]; a.wslot[r * P + id] = (uint8_t)slot[i]; }
+    }
   }
   if (lane == 0) {
     a.clock[r] = clock;
@@ -222,6 +341,14 @@ __global__ void __launch_bounds__(128) schedule_kernel(ScheduleArgs a) {
       a.q_last[r] = q_last; a.want_eval[r] = want;
     }
   }
+}
+
+inline cudaError_t launch_schedule(const ScheduleArgs& a, cudaStream_t stream) {
+  const int grid = (a.R + 3) / 4;
+  if (a.P <= 32) schedule_kernel<1><<<grid, 128, 0, stream>>>(a);
+  else if (a.P <= 64) schedule_kernel<2><<<grid, 128, 0, stream>>>(a);
+  else schedule_kernel<4><<<grid, 128, 0, stream>>>(a);
+  return cudaGetLastError();
 }
 
 // After the risk of the paused replicas is known: the rule of Section 6 / Algorithm 1.

@@ -429,8 +429,7 @@ sim_status sim_run(sim_handle* h, int64_t iters) {
     sa.K_cur = h->K_cur; sa.q_last = h->q_last; sa.want_eval = h->want_eval;
   }
   for (long long round = 0;; ++round) {
-  schedule_kernel<<<(h->R + 3) / 4, 128, 0, h->stream>>>(sa);
-  CUDA_TRY(h, cudaGetLastError());
+  CUDA_TRY(h, launch_schedule(sa, h->stream));
 
   if (h->prob.model != SIM_NONE) {
     NumericArgs a{};

@@ -69,3 +69,13 @@ def test_seed_uses_all_64_bits(B):
         assert_schedule_equal(sim.trace(), core.BulkSchedule("ksync", 4, 2, "exp", 1.0, 0.0, seed, 2).run(5))
         sim.close()
     assert not np.array_equal(out[0], out[1]) and not np.array_equal(out[0], out[2])
+
+
+@pytest.mark.parametrize("variant", list(core.VARIANTS))
+def test_more_workers_than_warp_lanes(B, variant):
+    """P = 40 and P = 128 workers (two / four per lane of the arrival kernel; 42 / 130 parameter versions):
+    parameters and losses of every model family against the oracle."""
+    run_case(B, inputs.make_lsq(600, 24, 0.1, 61), variant=variant, P=40, K=9, m=4, eta=0.02, R=3, J=40)
+    run_case(B, inputs.make_logistic(500, 12, 0.05, 62), variant=variant, P=128, K=17, m=3, eta=0.05, R=2, J=30, use_ref=False)
+    run_case(B, inputs.make_mixture(400, 20, 4, 0.5, 63, "softmax"), variant=variant, P=70, K=33, m=2, eta=0.05, R=2, J=20,
+             use_ref=False)

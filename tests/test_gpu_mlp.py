@@ -67,6 +67,14 @@ def test_mlp_variants_and_shapes(B, variant, d, H, C, m, K, P):
     run_mlp_case(B, data, w0, variant=variant, P=P, K=K, m=m, eta=0.02, R=3, J=12 if d > 1000 else 25, base=1)
 
 
+@pytest.mark.parametrize("variant", ["kasync", "kbatchasync"])
+def test_mlp_more_workers_than_warp_lanes(B, variant):
+    """P = 40: 42 parameter versions (and W1 shadows) per replica, two workers per lane in the arrival kernel."""
+    data = inputs.make_mixture(2048, 128, 3, 0.5, 99, "mlp2", 64)
+    w0 = inputs.mlp_init(128, 64, 3, 100)
+    run_mlp_case(B, data, w0, variant=variant, P=40, K=3, m=128, eta=0.02, R=2, J=20, base=2)
+
+
 def test_mlp_growing_K_and_resume(B):
     data = inputs.make_mixture(2048, 128, 4, 0.5, 97, "mlp2", 64)
     w0 = inputs.mlp_init(128, 64, 4, 98)

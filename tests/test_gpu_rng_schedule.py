@@ -63,6 +63,20 @@ def test_schedule_bit_exact(B, variant, P, K):
 
 
 @pytest.mark.parametrize("variant", list(core.VARIANTS))
+@pytest.mark.parametrize("P,K", [(33, 1), (33, 33), (48, 7), (64, 64), (64, 20), (65, 9), (100, 31), (128, 128), (128, 5)])
+def test_schedule_bit_exact_more_than_a_lane_per_worker(B, variant, P, K):
+    """P > 32: two or four workers per lane in the arrival kernel, up to 130 version-pool slots."""
+    check(B, variant, P, K, "shifted_exp", 0.9, 0.1, seed=15, R=7, J=60 if K > 40 else 120, base=3)
+
+
+@pytest.mark.parametrize("variant", list(core.VARIANTS))
+def test_schedule_wide_growing_K_ties_and_resume(B, variant):
+    check(B, variant, 80, 1, "exp", 1.0, 0.0, seed=16, R=5, J=150, K0=2, ti=1.5, chunks=[1, 49, 100])
+    check(B, variant, 40, 35, "shifted_exp", float("inf"), 0.5, R=2, J=6)          # all delays equal: ties by worker id
+    check(B, variant, 96, 12, "pareto2", 2.0, 1.0, seed=17, R=4, J=80)
+
+
+@pytest.mark.parametrize("variant", list(core.VARIANTS))
 def test_schedule_growing_K_and_resume(B, variant):
     check(B, variant, 8, 1, "shifted_exp", 2.0, 1.0, seed=6, R=20, J=260, K0=1, ti=30.0, chunks=[1, 59, 200])
     check(B, variant, 12, 1, "exp", 1.0, 0.0, seed=7, R=9, J=120, K0=3, ti=4.0)
@@ -86,7 +100,7 @@ def test_first_workload_schedule_all_replicas(B):
 def test_bad_arguments_are_refused(B):
     S = B.Simulation
     base = dict(P=4, K=2, variant="ksync", delay_kind="exp", mu=1.0, eta=0.1, m=4, seed=0, n_replicas=2)
-    for bad in (dict(P=0), dict(P=33), dict(K=0), dict(K=5), dict(m=0), dict(n_replicas=0), dict(mu=0.0),
+    for bad in (dict(P=0), dict(P=129), dict(K=0), dict(K=5), dict(m=0), dict(n_replicas=0), dict(mu=0.0),
                 dict(mu=float("nan")), dict(delay_kind="shifted_exp", shift=-1.0), dict(replica_base=2**32),
                 dict(delay_kind="pareto2", mu=3.0, shift=1.0), dict(delay_kind="pareto2", mu=2.0, shift=0.0)):
         with pytest.raises(B.SimError) as e:
