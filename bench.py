@@ -295,7 +295,7 @@ def main():
         host = {"model": "lsq", "X": Xp.numpy(), "y": yp.numpy()}
         kw = dict(P=wl.P, delay_kind=wl.delay_kind, mu=wl.mu, shift=wl.shift, eta=wl.eta, m=wl.m, seed=wl.seed,
                   n_replicas=R, replica_base=rank * R, iters=U, want=("t", "loss"))
-        e2e_steps = max(1, min(args.steps, 5))
+        e2e_steps = max(1, min(args.steps, 10))
         sweep_host(host, wl.runs, **kw)
         barrier()
         t0 = time.perf_counter()

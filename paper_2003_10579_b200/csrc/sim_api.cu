@@ -74,6 +74,7 @@ struct sim_handle {
   int* K_cur = nullptr; int* want_eval = nullptr; int* remaining = nullptr;
   TraceBuffers tr;
   bool poisoned = false;
+  bool in_arena = false;      // buffers come from the creating thread's DeviceArena and are not freed one by one
   mutable std::string last_error;
 };
 
@@ -92,11 +93,43 @@ sim_status fail(const sim_handle* h, sim_status st, const std::string& msg) {
                   std::string(#expr) + ": " + cudaGetErrorString(e_));                      \
   } while (0)
 
+// Device memory for many short-lived handles at once (sim_sweep_host): buffers are carved out of a few
+// large chunks instead of one cudaMalloc / cudaFree each (a cudaFree waits for the whole device).  While
+// a host thread has an arena installed, every handle it creates takes its buffers from it and frees
+// none of them; the arena's owner releases the chunks after the handles are gone.
+struct DeviceArena {
+  std::vector<void*> chunks;
+  char* cur = nullptr;
+  size_t left = 0;
+  cudaError_t take(void** p, size_t bytes) {
+    bytes = (bytes + 255) & ~(size_t)255;
+    if (bytes > left) {
+      const size_t chunk = bytes > ((size_t)64 << 20) ? bytes : ((size_t)64 << 20);
+      void* c = nullptr;
+      const cudaError_t e = cudaMalloc(&c, chunk);
+      if (e != cudaSuccess) return e;
+      chunks.push_back(c);
+      cur = static_cast<char*>(c);
+      left = chunk;
+    }
+    *p = cur;
+    cur += bytes;
+    left -= bytes;
+    return cudaSuccess;
+  }
+  void release() {
+    for (void* c : chunks) cudaFree(c);
+    chunks.clear(); cur = nullptr; left = 0;
+  }
+};
+thread_local DeviceArena* t_arena = nullptr;
+
 template <typename T>
 cudaError_t dev_alloc(T** p, size_t count, cudaStream_t st, bool zero = true) {
   *p = nullptr;
   if (count == 0) return cudaSuccess;
-  cudaError_t e = cudaMalloc(reinterpret_cast<void**>(p), count * sizeof(T));
+  cudaError_t e = t_arena ? t_arena->take(reinterpret_cast<void**>(p), count * sizeof(T))
+                          : cudaMalloc(reinterpret_cast<void**>(p), count * sizeof(T));
   if (e != cudaSuccess) { *p = nullptr; return e; }
   if (zero) e = cudaMemsetAsync(*p, 0, count * sizeof(T), st);
   return e;
@@ -156,7 +189,7 @@ sim_status regrow(sim_handle* h, T** buf, size_t per_update, long long new_cap, 
                                   (size_t)h->n_updates * per_update * sizeof(T), h->R,
                                   cudaMemcpyDeviceToDevice, h->stream));
   }
-  if (*buf) { CUDA_TRY(h, cudaStreamSynchronize(h->stream)); cudaFree(*buf); }
+  if (*buf && !h->in_arena) { CUDA_TRY(h, cudaStreamSynchronize(h->stream)); cudaFree(*buf); }
   *buf = nb;
   return SIM_OK;
 }
@@ -236,9 +269,10 @@ sim_status device_error(const sim_handle* h) {
 }
 
 void free_all(sim_handle* h) {
+  mlp_scratch_free(h->mlp);
+  if (h->in_arena) return;          // the arena's owner frees the chunks
   cudaFree(h->s); cudaFree(h->tau); cudaFree(h->f); cudaFree(h->wslot); cudaFree(h->cur_slot);
   cudaFree(h->begin_slot); cudaFree(h->clock); cudaFree(h->w_state); cudaFree(h->pool); cudaFree(h->err);
-  mlp_scratch_free(h->mlp);
   cudaFree(h->eval_partial); cudaFree(h->F0); cudaFree(h->Fcur); cudaFree(h->done); cudaFree(h->run_j0);
   cudaFree(h->run_iters); cudaFree(h->q_last); cudaFree(h->K_cur); cudaFree(h->want_eval); cudaFree(h->remaining);
   cudaFree(h->tr.t); cudaFree(h->tr.loss); cudaFree(h->tr.dist2); cudaFree(h->tr.K_used);
@@ -321,6 +355,7 @@ sim_status sim_create(const sim_problem* problem, int32_t P, int32_t K, sim_vari
   }
 
   sim_handle* h = new (std::nothrow) sim_handle();
+  if (h) h->in_arena = t_arena != nullptr;
   if (!h) return fail(nullptr, SIM_ERR_ALLOC, "host allocation failed");
   h->prob = prob; h->P = P; h->K = K; h->variant = (int)variant; h->delay = delay; h->eta = eta;
   h->m = m; h->seed = seed; h->R = n_replicas; h->replica_base = (uint32_t)replica_base;
@@ -704,6 +739,8 @@ sim_status sim_sweep_host(const sim_problem* problem, int32_t P, int32_t n_runs,
     return true;
   };
   const size_t RJ = (size_t)n_replicas * (size_t)iters;
+  DeviceArena arena;                    // the runs' state, parameters and traces: a few chunks instead of hundreds of buffers
+  t_arena = &arena;
   do {
     void *X, *y, *lab, *wr, *dw0;
     if (!up(problem->X, (size_t)dp.n * dp.d * 4, &X)) break;
@@ -740,7 +777,9 @@ sim_status sim_sweep_host(const sim_problem* problem, int32_t P, int32_t n_runs,
     if (hs[i]) sim_destroy(hs[i]);
     if (streams[i]) cudaStreamDestroy(streams[i]);
   }
+  t_arena = nullptr;
   cudaDeviceSynchronize();
+  arena.release();
   for (void* p : owned) cudaFree(p);
   if (st != SIM_OK) return fail(nullptr, st, "sim_sweep_host: " + msg);
   return SIM_OK;
