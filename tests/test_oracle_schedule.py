@@ -30,7 +30,7 @@ def z_ok(sample, mean, var, z=4.5):
 
 # ---- Lemma 1 / Appendix B.1: K-sync, T = X_{K:P}; Exp: (H_P - H_{P-K})/mu, variance sum 1/(i mu)^2
 @pytest.mark.parametrize("P,K,mu,shift", [(4, 2, 1.0, 0.0), (16, 5, 2.0, 0.0), (16, 16, 1.0, 0.0),
-                                          (8, 3, 2.0, 1.0), (16, 1, 1.0, 0.5)])
+                                          (8, 3, 2.0, 1.0), (16, 1, 1.0, 0.5), (64, 40, 1.0, 0.0), (128, 9, 1.5, 0.25)])
 def test_ksync_mean_and_variance(P, K, mu, shift):
     kind = "shifted_exp" if shift else "exp"
     T = iteration_times(bulk("ksync", P, K, kind, mu, shift, seed=3, R=64, J=400))
@@ -57,7 +57,7 @@ def test_ksync_each_worker_selected_with_frequency_K_over_P():
 
 
 # ---- Lemma 2 / Appendix B.2: K-batch-sync; Exp: T ~ Erlang(K, P mu)
-@pytest.mark.parametrize("P,K,mu", [(4, 2, 1.0), (16, 7, 1.0), (16, 16, 3.0)])
+@pytest.mark.parametrize("P,K,mu", [(4, 2, 1.0), (16, 7, 1.0), (16, 16, 3.0), (100, 33, 1.0)])
 def test_kbatchsync_erlang(P, K, mu):
     T = iteration_times(bulk("kbatchsync", P, K, "exp", mu, seed=6, R=64, J=400))
     assert z_ok(T, K / (P * mu), K / (P * mu) ** 2)
@@ -75,7 +75,7 @@ def test_kbatchsync_shifted_bound():
 
 
 # ---- Lemma 3: K-async; Exp: equality with E[X_{K:P}]; new-longer-than-used: upper bound
-@pytest.mark.parametrize("P,K", [(8, 1), (8, 3), (16, 8), (32, 4)])
+@pytest.mark.parametrize("P,K", [(8, 1), (8, 3), (16, 8), (32, 4), (96, 20)])
 def test_kasync_exp_mean(P, K):
     T = iteration_times(bulk("kasync", P, K, seed=8, R=64, J=600))
     mean = H(P) - H(P - K)
