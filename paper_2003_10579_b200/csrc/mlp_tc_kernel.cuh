@@ -106,7 +106,7 @@ inline __host__ __device__ TcLayout tc_forward_layout(int H) {
 }
 
 __global__ void __launch_bounds__(TC_THREADS, 1)
-mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, MlpArgs g) {
+mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmW, MlpArgs g) {
   const NumericArgs& a = g.na;
   const MlpScratch& sc = g.sc;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -691,15 +691,14 @@ inline bool tc_make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-struct MlpMaps { CUtensorMap tmX, tmW, tmD; bool ready = false; };
+struct MlpMaps { CUtensorMap tmW, tmD; bool ready = false; };
 
 inline cudaError_t run_mlp(NumericArgs& a, MlpScratch& s, MlpMaps& maps, int P, cudaStream_t stream, const char** why) {
   *why = nullptr;
   cudaError_t e;
   const int n_halves = s.H > 256 ? 2 : 1;
   if (!maps.ready) {
-    if (!tc_make_map(&maps.tmX, s.Xq, (uint64_t)s.n, (uint64_t)s.d, TC_BK, 1) ||
-        !tc_make_map(&maps.tmW, s.W1qT, (uint64_t)s.R * s.n_slots * (s.d / TC_BK) * s.H, (uint64_t)TC_BK, TC_BK, (uint32_t)(s.H / n_halves)) ||
+    if (!tc_make_map(&maps.tmW, s.W1qT, (uint64_t)s.R * s.n_slots * (s.d / TC_BK) * s.H, (uint64_t)TC_BK, TC_BK, (uint32_t)(s.H / n_halves)) ||
         !tc_make_map(&maps.tmD, s.D1q, (uint64_t)s.R * s.Kmax * s.m, (uint64_t)s.H, 64, 64)) {
       *why = "mlp: could not encode the TMA tensor maps";
       return cudaSuccess;
@@ -721,7 +720,7 @@ inline cudaError_t run_mlp(NumericArgs& a, MlpScratch& s, MlpMaps& maps, int P, 
   for (long long u = 0; u < a.iters; ++u) {
     g.j = a.j0 + u;
     mlp_rows_kernel<<<a.R * s.Kmax, 128, 0, stream>>>(g);
-    mlp_forward_tc_kernel<<<a.R * s.Kmax * mtiles, TC_THREADS, L.total, stream>>>(maps.tmX, maps.tmW, g);
+    mlp_forward_tc_kernel<<<a.R * s.Kmax * mtiles, TC_THREADS, L.total, stream>>>(maps.tmW, g);
     mlp_head_kernel<<<a.R * (s.H / 32), MLP_HEAD_THREADS, 0, stream>>>(g);
     mlp_dw1_tc_kernel<<<dw1_grid, DW1_THREADS, LD.total, stream>>>(maps.tmD, g);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;

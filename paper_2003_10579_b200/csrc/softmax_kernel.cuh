@@ -41,6 +41,19 @@ __device__ __forceinline__ void warp_transpose_reduce(float (&v)[32], int lane) 
   transpose_reduce_step<1, 2>(v, lane);
 }
 
+// Two fp32 FMAs in one instruction (each half rounds like fmaf): halves the issue slots of the two products.
+__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+  return d;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+
 template <int CHUNKS, int CP, bool ASYNC>
 __global__ void __launch_bounds__(SMX_NT) softmax_kernel(NumericArgs a) {
   constexpr int NT = SMX_NT, NW = NT / 32, T = SMX_T, E = 4 * CHUNKS, CH = CP / 2;
@@ -126,11 +139,11 @@ __global__ void __launch_bounds__(SMX_NT) softmax_kernel(NumericArgs a) {
   __syncthreads();
   if (my_iters <= 0) return;
 
-  float G[CP][E];
+  uint64_t G[CP][E / 2];      // pairs of adjacent columns
 #pragma unroll
   for (int c = 0; c < CP; ++c)
 #pragma unroll
-    for (int e = 0; e < E; ++e) G[c][e] = 0.f;
+    for (int e = 0; e < E / 2; ++e) G[c][e] = 0ull;
   float loss_acc = 0.f;      // meaningful in the row-leader threads of the softmax stage
   long long j = my_j0;
   bool failed = false;
@@ -152,15 +165,15 @@ __global__ void __launch_bounds__(SMX_NT) softmax_kernel(NumericArgs a) {
     }
 
     // ---- x of own columns -> registers; label of the row this thread serves in the softmax stage ----
-    float x[T][E];
+    uint64_t x[T][E / 2];      // pairs of adjacent columns, as the 16-byte loads deliver them
 #pragma unroll
     for (int c = 0; c < CHUNKS; ++c) {
       const int ci = tid + NT * c;
 #pragma unroll
       for (int q = 0; q < T; ++q) {
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (ci < d4 && q < ti.rows) v = reinterpret_cast<const float4*>(tile + (size_t)q * d)[ci];
-        x[q][4 * c] = v.x; x[q][4 * c + 1] = v.y; x[q][4 * c + 2] = v.z; x[q][4 * c + 3] = v.w;
+        ulonglong2 v = make_ulonglong2(0ull, 0ull);
+        if (ci < d4 && q < ti.rows) v = reinterpret_cast<const ulonglong2*>(tile + (size_t)q * d)[ci];
+        x[q][2 * c] = v.x; x[q][2 * c + 1] = v.y;
       }
     }
     int label = 0;
@@ -183,11 +196,14 @@ __global__ void __launch_bounds__(SMX_NT) softmax_kernel(NumericArgs a) {
               const float4 w = reinterpret_cast<const float4*>(W_s + (size_t)cls * d)[ci];
 #pragma unroll
               for (int q = 0; q < T; ++q) {
+                float x0, x1, x2, x3;
+                unpack2(x[q][2 * c], x0, x1);
+                unpack2(x[q][2 * c + 1], x2, x3);
                 float acc = v[q * CH + cc];
-                acc = fmaf(x[q][4 * c], w.x, acc);
-                acc = fmaf(x[q][4 * c + 1], w.y, acc);
-                acc = fmaf(x[q][4 * c + 2], w.z, acc);
-                acc = fmaf(x[q][4 * c + 3], w.w, acc);
+                acc = fmaf(x0, w.x, acc);
+                acc = fmaf(x1, w.y, acc);
+                acc = fmaf(x2, w.z, acc);
+                acc = fmaf(x3, w.w, acc);
                 v[q * CH + cc] = acc;
               }
             }
@@ -247,8 +263,9 @@ __global__ void __launch_bounds__(SMX_NT) softmax_kernel(NumericArgs a) {
           for (int k = 0; k < 4; ++k) {
             const int cls = 4 * c4 + k;
             if (cls < CP) {
+              const uint64_t dd2 = pack2(dl[k], dl[k]);
 #pragma unroll
-              for (int e = 0; e < E; ++e) G[cls][e] = fmaf(dl[k], x[q][e], G[cls][e]);
+              for (int e = 0; e < E / 2; ++e) G[cls][e] = ffma2(dd2, x[q][e], G[cls][e]);
             }
           }
         }
@@ -268,10 +285,13 @@ __global__ void __launch_bounds__(SMX_NT) softmax_kernel(NumericArgs a) {
           for (int cls = 0; cls < CP; ++cls) {
             if (cls < C) {
               float4 w = reinterpret_cast<const float4*>(w_from + (size_t)cls * d)[ci];
-              w.x = fmaf(-scale, G[cls][4 * c], w.x);
-              w.y = fmaf(-scale, G[cls][4 * c + 1], w.y);
-              w.z = fmaf(-scale, G[cls][4 * c + 2], w.z);
-              w.w = fmaf(-scale, G[cls][4 * c + 3], w.w);
+              float g0, g1, g2, g3;
+              unpack2(G[cls][2 * c], g0, g1);
+              unpack2(G[cls][2 * c + 1], g2, g3);
+              w.x = fmaf(-scale, g0, w.x);
+              w.y = fmaf(-scale, g1, w.y);
+              w.z = fmaf(-scale, g2, w.z);
+              w.w = fmaf(-scale, g3, w.w);
               reinterpret_cast<float4*>(w_to + (size_t)cls * d)[ci] = w;
               if (a.w_ref) {
                 const float4 wr = reinterpret_cast<const float4*>(a.w_ref + (size_t)cls * d)[ci];
@@ -279,8 +299,7 @@ __global__ void __launch_bounds__(SMX_NT) softmax_kernel(NumericArgs a) {
                 dd = fmaf(e0, e0, dd); dd = fmaf(e1, e1, dd); dd = fmaf(e2, e2, dd); dd = fmaf(e3, e3, dd);
               }
             }
-#pragma unroll
-            for (int e = 0; e < 4; ++e) G[cls][4 * c + e] = 0.f;
+            G[cls][2 * c] = 0ull; G[cls][2 * c + 1] = 0ull;
           }
         }
       }
