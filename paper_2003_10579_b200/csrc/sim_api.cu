@@ -11,6 +11,7 @@
 
 #include "linear_kernel.cuh"
 #include "softmax_kernel.cuh"
+#include "softmax_tm_kernel.cuh"
 #include "mlp_tc_kernel.cuh"
 #include "eval_kernel.cuh"
 
@@ -483,7 +484,7 @@ sim_status sim_run(sim_handle* h, int64_t iters) {
     switch (h->prob.model) {
       case SIM_LSQ: case SIM_LOGISTIC: st = run_linear1(h, a); break;
       case SIM_SOFTMAX:
-        ce = run_softmax(a, h->tune_stages, h->stream, &why);
+        ce = run_softmax_any(a, h->tune_stages, h->stream, &why);
         st = why ? fail(h, SIM_ERR_ARG, why) : SIM_OK;
         break;
       case SIM_MLP2:
