@@ -335,6 +335,7 @@ __global__ void __launch_bounds__(128 * NG) softmax_tm_kernel(NumericArgs a) {
     if (warp == 0 && it >= 1) issue_tile(it + 1);          // into the stage of tile it - 1
 
     // ---- softmax stage: thread (sq, sc) owns logit (row sq, class sc) ----
+    float loss_term = 0.f, loss_s1 = 0.f;
     if (st_tid >= 0) {
       float z = -INFINITY;
       const bool live = sc < C && sq < ti.rows;
@@ -359,17 +360,19 @@ __global__ void __launch_bounds__(128 * NG) softmax_tm_kernel(NumericArgs a) {
       float sexcl = ez;
 #pragma unroll
       for (int off = 8; off > 0; off >>= 1) sexcl += __shfl_xor_sync(0xFFFFFFFFu, sexcl, off);
-      const float ssum = 1.f + sexcl;
+      const float inv = __frcp_rn(1.f + sexcl);   // one correctly rounded reciprocal instead of a division per case
       const float zlab = __shfl_sync(0xFFFFFFFFu, z, (lane & 16) + label);
       float dl = 0.f;
       if (live) {
-        if (is_max) dl = sc == label ? -sexcl / ssum : 1.f / ssum;
-        else dl = ez / ssum - (sc == label ? 1.f : 0.f);
+        if (is_max) dl = sc == label ? -sexcl * inv : inv;
+        else dl = ez * inv - (sc == label ? 1.f : 0.f);
       }
       if (sc < CP) reinterpret_cast<float2*>(delta_s)[sq * CP + sc] = make_float2(dl, dl);
-      if (sc == 0 && sq < ti.rows) loss_acc += log1pf(sexcl) + (zmax - zlab);
+      loss_term = (sc == 0 && sq < ti.rows) ? zmax - zlab : 0.f;
+      loss_s1 = (sc == 0 && sq < ti.rows) ? sexcl : 0.f;
     }
     __syncthreads();   // (B)
+    if (st_tid >= 0) loss_acc += log1pf(loss_s1) + loss_term;   // off the path the other warps wait on
 
     // ---- G += D^T X over own pairs ----
     // (every row of the tile: the softmax stage wrote zeros for the rows a ragged tile does not have)
