@@ -204,10 +204,12 @@ __global__ void __launch_bounds__(NT) linear1_kernel(NumericArgs a) {
   // ---- producer (warp 0): stage tiles of rows ahead of the arithmetic ----
   ScheduleWalk walk;
   walk.done = true;
-  auto issue_tile = [&](long long tile_no) {
+  int prod_st = 0;
+  auto issue_tile = [&](long long) {
     // called by all lanes of warp 0; the stage's previous contents have been consumed
     if (walk.done) return;
-    const int st = (int)(tile_no % S);
+    const int st = prod_st;   // tiles are issued in order: a counter, not a 64-bit modulo per tile
+    if (++prod_st == S) prod_st = 0;
     const uint32_t bar = smem_addr(&full[st]);
     const int rows = min(T, m - walk.k * T);
     if (walk.k == 0) {   // a new task: its m sample rows are drawn once, 32 at a time (only this warp uses the table)
@@ -253,9 +255,9 @@ __global__ void __launch_bounds__(NT) linear1_kernel(NumericArgs a) {
   float loss_acc = 0.f;
   long long j = my_j0;
   bool failed = false;
-  for (long long it = 0;; ++it) {
-    const int st = (int)(it % S);
-    const uint32_t parity = (uint32_t)((it / S) & 1);
+  int st = 0;             // stage and phase parity of tile `it`, kept as counters (it % S and it / S are 64-bit divisions)
+  uint32_t parity = 0;
+  for (long long it = 0;; ++it, parity ^= (uint32_t)(st + 1 == S), st = (st + 1 == S ? 0 : st + 1)) {
     if (!mbar_wait(smem_addr(&full[st]), parity)) { failed = true; break; }
     const TileInfo ti = info_s[st];
     const float* tile = rows_s + (size_t)st * T * d;
