@@ -443,6 +443,13 @@ __device__ __forceinline__ void bulk_s2g(void* dst, uint32_t src, uint32_t bytes
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// Position in a ring of n slots: slot and phase parity of use number u, stepped as counters (u % n and u / n with a
+// run-time n and a 64-bit u are a division subroutine each, on the critical path of single-thread roles).
+struct RingPos {
+  int s;
+  uint32_t ph;
+  __device__ __forceinline__ void step(int n, int by = 1) { s += by; if (s >= n) { s -= n; ph ^= 1u; } }
+};
 
 __global__ void __launch_bounds__(DW1_THREADS, 1)
 mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
@@ -496,12 +503,12 @@ mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
   if (warp == 0) {
     // ---- B producer: delta1 rows of 64 samples, Hn/64 boxes of 64 x 64 ----
     if (lane == 0) {
-      long long it = 0;
+      RingPos rp{0, 0u};
       for (int t = blockIdx.x; t < n_tiles && !failed; t += gridDim.x) {
         const int r = tile_r(t), part = t % parts, nk = tile_nk(t);
-        for (int kc = 0; kc < nk; ++kc, ++it) {
-          const int s = (int)(it % S);
-          if (!mbar_wait(empty_bar(s), (uint32_t)(((it / S) & 1) ^ 1))) { failed = true; break; }
+        for (int kc = 0; kc < nk; ++kc, rp.step(S)) {
+          const int s = rp.s;
+          if (!mbar_wait(empty_bar(s), rp.ph ^ 1u)) { failed = true; break; }
           const uint32_t Bs = base_addr + (uint32_t)s * L.stage_bytes + TC_A_BYTES;
           const int row0 = (int)((size_t)r * sc.Kmax * m + (size_t)kc * TC_BK);
           mbar_arrive_expect_tx(full_bar(s), (uint32_t)(Hn * 128));
@@ -514,15 +521,15 @@ mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
     // ---- MMA issuer ----
     const uint32_t idesc = tc_idesc(Hn, 1, 1);
     const uint32_t lbo = ATOM, sbo = 1024u;   // next 64 MN elements: one atom block on; next 8 samples: 1024 B on
-    long long it = 0;
+    RingPos rp{0, 0u};
     int i = 0;
     for (int t = blockIdx.x; t < n_tiles && !failed; t += gridDim.x, ++i) {
       const int nk = tile_nk(t), buf = i & 1;
       if (!mbar_wait(acc_empty(buf), (uint32_t)(((i >> 1) & 1) ^ 1))) { failed = true; break; }
       tc_fence_after();
-      for (int kc = 0; kc < nk; ++kc, ++it) {
-        const int s = (int)(it % S);
-        if (!mbar_wait(full_bar(s), (uint32_t)((it / S) & 1))) { failed = true; break; }
+      for (int kc = 0; kc < nk; ++kc, rp.step(S)) {
+        const int s = rp.s;
+        if (!mbar_wait(full_bar(s), rp.ph)) { failed = true; break; }
         tc_fence_after();
         if (lane == 0) {
           const uint32_t As = base_addr + (uint32_t)s * L.stage_bytes, Bs = As + TC_A_BYTES;
@@ -545,19 +552,21 @@ mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
     const int p = tid - 64, piece = p & 15, k0 = p >> 4;
     const int lag = S > 2 ? S - 2 : 1;
     long long it = 0, signalled = 0;
-    auto signal = [&](long long which) {
+    RingPos rp{0, 0u}, sig{0, 0u};
+    auto signal = [&](long long) {      // stages are signalled in order
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      mbar_arrive(full_bar((int)(which % S)));
+      mbar_arrive(full_bar(sig.s));
+      sig.step(S);
     };
     for (int t = blockIdx.x; t < n_tiles && !failed; t += gridDim.x) {
       const int r = tile_r(t), slab = (t / parts) % slabs, nk = tile_nk(t);
       const int* rows = sc.rows_tab + (size_t)r * sc.Kmax * m;
-      for (int kc = 0; kc < nk; ++kc, ++it) {
-        const int s = (int)(it % S);
+      for (int kc = 0; kc < nk; ++kc, ++it, rp.step(S)) {
+        const int s = rp.s;
         int rid[8];                     // issued before the wait: the ring is usually full, the latency hides there
 #pragma unroll
         for (int i = 0; i < 8; ++i) rid[i] = rows[kc * TC_BK + k0 + 8 * i];
-        if (!mbar_wait(empty_bar(s), (uint32_t)(((it / S) & 1) ^ 1))) { failed = true; break; }
+        if (!mbar_wait(empty_bar(s), rp.ph ^ 1u)) { failed = true; break; }
         const uint32_t As = base_addr + (uint32_t)s * L.stage_bytes + (uint32_t)(piece >> 3) * ATOM;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
@@ -583,7 +592,7 @@ mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
     // shadow element (k, n) lives at [(k / 64) * H + n] * 64 + k % 64: in the staging copy of a block,
     // [k / 64][n - first column][k % 64]
     __nv_bfloat16* qrow = reinterpret_cast<__nv_bfloat16*>(qstage) + (rloc >> 6) * 2048 + (rloc & 63);
-    long long n = grp;                                  // running number of the block among all blocks of this CTA
+    RingPos wp{grp % NB, (uint32_t)((grp / NB) & 1)};   // ring position of this group's running block number grp, grp + 2, ...
     int i = 0;
     for (int t = blockIdx.x; t < n_tiles && !failed; t += gridDim.x, ++i) {
       const int r = tile_r(t), slab = (t / parts) % slabs, part = t % parts, buf = i & 1;
@@ -593,9 +602,9 @@ mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
       float* wn = a.pool + ((size_t)r * a.n_slots + fresh) * a.slot_stride + (((size_t)slab * (H >> 5) + ((part * Hn) >> 5)) << 12);
       __nv_bfloat16* wq = sc.W1qT + ((size_t)r * sc.n_slots + fresh) * dH + ((size_t)(2 * slab) * H + part * Hn) * 64;
       const uint32_t trow = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * Hn);
-      for (int b = grp; b < nb; b += 2, n += 2) {
-        const int s = (int)(n % NB);
-        bool ok = mbar_wait(wfull(s), (uint32_t)((n / NB) & 1));
+      for (int b = grp; b < nb; b += 2, wp.step(NB, 2)) {
+        const int s = wp.s;
+        bool ok = mbar_wait(wfull(s), wp.ph);
         if (ok && b == grp) ok = mbar_wait(acc_full(buf), (uint32_t)((i >> 1) & 1));
         if (!ok) fail_s[grp] = 1;
         group_barrier(1 + grp, 128);                    // the four warps give up together or not at all
@@ -643,12 +652,12 @@ mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
                (((size_t)slab * (H >> 5) + ((part * Hn) >> 5)) << 12);
       };
       const int nb = Hn / 32;
-      long long n = 0;
+      RingPos wp{0, 0u};
       for (int t = blockIdx.x; t < n_tiles && !failed; t += gridDim.x) {
         const float* src = tile_src(t);
-        for (int b = 0; b < nb; ++b, ++n) {
-          const int s = (int)(n % NB);
-          if (!mbar_wait(wempty(s), (uint32_t)(((n / NB) & 1) ^ 1))) { failed = true; break; }
+        for (int b = 0; b < nb; ++b, wp.step(NB)) {
+          const int s = wp.s;
+          if (!mbar_wait(wempty(s), wp.ph ^ 1u)) { failed = true; break; }
           mbar_arrive_expect_tx(wfull(s), DW1_WBLOCK);
           bulk_g2s(base_addr + L.off_w + s * DW1_WBLOCK, src + (size_t)b * 4096, DW1_WBLOCK, wfull(s));
         }
