@@ -30,7 +30,7 @@
 #define SMX_TM_NG 3
 #endif
 #ifndef SMX_TM_TG
-#define SMX_TM_TG 2
+#define SMX_TM_TG 3
 #endif
 #ifndef SMX_TM_DB
 #define SMX_TM_DB 0
@@ -130,8 +130,8 @@ __global__ void __launch_bounds__(128 * NG) softmax_tm_kernel(NumericArgs a) {
   constexpr int NT = 128 * NG, NW = 4 * NG, T = NG * TG, CP = SMT_CP, WC = SMT_WC, OWN = KP * WC, NV = TG * CP;
   constexpr int DS = 2 * NT * KP;      // floats between row slots: every thread can read its pairs without a bounds test
   static_assert(NG * OWN <= (int)SMT_TMEM_COLS, "the parameters must fit the allocated columns");
-  static_assert(16 * T <= NT && T <= 32 && NV <= 32, "tile shape");
-  static_assert((16 * T) % 32 == 0, "the softmax stage shuffles with a full mask: it must be made of whole warps");
+  constexpr int SW = (16 * T + 31) / 32;   // warps of the softmax stage: whole warps, it shuffles with a full mask
+  static_assert(32 * SW <= NT && T <= 32 && NV <= 32, "tile shape");
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int grp = tid >> 7, L = tid & 127;
   const int r = blockIdx.x;
@@ -255,7 +255,7 @@ __global__ void __launch_bounds__(128 * NG) softmax_tm_kernel(NumericArgs a) {
   long long j = my_j0;
   bool failed = false;
   int cur_slot = ASYNC ? (int)a.begin_slot[r] : 0;
-  const int st_tid = tid - (NT - 16 * T);          // the last warps serve the softmax stage (warp 0 is the producer)
+  const int st_tid = tid - (NT - 32 * SW);         // the last warps serve the softmax stage (warp 0 is the producer)
   const int sq = st_tid >> 4, sc = st_tid & 15;    // 16 lanes per row
   const int red_idx = tm_reduce_index<NV>(lane);
 
@@ -367,7 +367,7 @@ __global__ void __launch_bounds__(128 * NG) softmax_tm_kernel(NumericArgs a) {
         if (is_max) dl = sc == label ? -sexcl * inv : inv;
         else dl = ez * inv - (sc == label ? 1.f : 0.f);
       }
-      if (sc < CP) reinterpret_cast<float2*>(delta_s)[sq * CP + sc] = make_float2(dl, dl);
+      if (sc < CP && sq < T) reinterpret_cast<float2*>(delta_s)[sq * CP + sc] = make_float2(dl, dl);
       loss_term = (sc == 0 && sq < ti.rows) ? zmax - zlab : 0.f;
       loss_s1 = (sc == 0 && sq < ti.rows) ? sexcl : 0.f;
     }
@@ -435,7 +435,7 @@ __global__ void __launch_bounds__(128 * NG) softmax_tm_kernel(NumericArgs a) {
       if (ASYNC) cur_slot = ti.fresh;
       dd = warp_sum(dd);
       if (lane == 0) misc_s[warp] = dd;
-      if (st_tid >= 0 && sc == 0) lossrow_s[sq] = loss_acc;
+      if (st_tid >= 0 && sc == 0 && sq < T) lossrow_s[sq] = loss_acc;
     }
     if (reload) load_w(a.pool + ((size_t)r * a.n_slots + ti.next_snap) * np);   // the next task's snapshot (own elements only)
     if (last_of_update || reload) {
