@@ -172,7 +172,7 @@ __global__ void __launch_bounds__(NT) linear1_kernel(NumericArgs a) {
   uint64_t* full = reinterpret_cast<uint64_t*>(smem);
   TileInfo* info_s = reinterpret_cast<TileInfo*>(smem + 8 * S);
   uint32_t* y_s = reinterpret_cast<uint32_t*>(info_s + S);
-  float* red_s = reinterpret_cast<float*>(y_s + S * T);
+  float* red_s = reinterpret_cast<float*>((reinterpret_cast<uintptr_t>(y_s + S * T) + 15) & ~(uintptr_t)15);   // read as vectors
   float* misc_s = red_s + 2 * NW * T;
   const size_t head = (size_t)((unsigned char*)(misc_s + NW) - smem);
   float* rows_s = reinterpret_cast<float*>(smem + ((head + 127) & ~(size_t)127));
@@ -310,14 +310,32 @@ __global__ void __launch_bounds__(NT) linear1_kernel(NumericArgs a) {
     if (warp == 0) issue_tile(it + S - 1);
 
     // ---- a_q = dl/dz and the loss ----
-    float aq[T];
+    float aq[T], zq[T];
+#pragma unroll
+    for (int q = 0; q < T; ++q) zq[q] = 0.f;
+    {   // the warps' partial sums of all T rows, a vector load per warp
+      constexpr int V = T % 4 == 0 ? 4 : 2;
+      static_assert(T % 2 == 0, "tile rows are read in pairs");
+      const float* rp = red_s + (it & 1) * NW * T;
+#pragma unroll
+      for (int w = 0; w < NW; ++w) {
+#pragma unroll
+        for (int q = 0; q < T; q += V) {
+          if (V == 4) {
+            const float4 v = *reinterpret_cast<const float4*>(rp + w * T + q);
+            zq[q] += v.x; zq[q + 1] += v.y; zq[q + 2] += v.z; zq[q + 3] += v.w;
+          } else {
+            const float2 v = *reinterpret_cast<const float2*>(rp + w * T + q);
+            zq[q] += v.x; zq[q + 1] += v.y;
+          }
+        }
+      }
+    }
 #pragma unroll
     for (int q = 0; q < T; ++q) {
       aq[q] = 0.f;
       if (q < ti.rows) {
-        float z = 0.f;
-#pragma unroll
-        for (int w = 0; w < NW; ++w) z += red_s[((it & 1) * NW + w) * T + q];
+        const float z = zq[q];
         const uint32_t yraw = y_s[st * T + q];
         if (a.model == M_LSQ) {
           const float res = z - __uint_as_float(yraw);
@@ -327,11 +345,11 @@ __global__ void __launch_bounds__(NT) linear1_kernel(NumericArgs a) {
           const float b = (float)(int)yraw;
           const float ez = expf(-fabsf(z));
           // sigmoid(z) - b without cancellation: sigma - 1 is formed directly for b = 1
-          const float inv = 1.f / (1.f + ez);
+          const float inv = __frcp_rn(1.f + ez);   // the correctly rounded 1 / (1 + ez), without the division's slow path
           const float sig = z >= 0.f ? inv : ez * inv;
           const float sig_m1 = z >= 0.f ? -ez * inv : -inv;
           aq[q] = b != 0.f ? sig_m1 : sig;
-          loss_acc += fmaxf(z, 0.f) + log1pf(ez) - b * z;
+          if (tid == 0) loss_acc += fmaxf(z, 0.f) + log1pf(ez) - b * z;   // only thread 0 records the loss
         }
       }
     }
@@ -410,7 +428,7 @@ __global__ void __launch_bounds__(NT) linear1_kernel(NumericArgs a) {
 
 // shared-memory bytes of linear1_kernel for a given shape
 inline size_t linear1_smem_bytes(int NT, int T, int S, int d, int m) {
-  size_t head = 8 * (size_t)S + sizeof(TileInfo) * (size_t)S + 4 * (size_t)S * T + 4 * (size_t)2 * (NT / 32) * T + 4 * (size_t)(NT / 32);
+  size_t head = 8 * (size_t)S + sizeof(TileInfo) * (size_t)S + 4 * (size_t)S * T + 16 + 4 * (size_t)2 * (NT / 32) * T + 4 * (size_t)(NT / 32);
   head = (head + 127) & ~(size_t)127;
   return head + (size_t)S * T * d * 4 + (size_t)m * 4;
 }
