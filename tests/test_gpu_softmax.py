@@ -24,6 +24,17 @@ def test_softmax_variants_and_shapes(B, variant, d, C, m, K, P):
              base=2, chunks=[10], use_ref=False)
 
 
+@pytest.mark.parametrize("variant", ["ksync", "kbatchasync"])
+@pytest.mark.parametrize("d,C,m", [(3072, 10, 21), (1540, 7, 9), (1536, 16, 6), (64, 3, 8)])
+def test_softmax_distance_to_a_reference(B, variant, d, C, m):
+    """`dist2` = |W_{j+1} - W_ref|^2 of every update, for both softmax kernels (tensor-memory parameters up to
+    10 classes, shared-memory parameters beyond), ragged tiles included."""
+    data = inputs.make_mixture(1500, d, C, 0.5 if d < 1000 else 0.05, 92)
+    data["w_star"] = (0.01 * np.random.default_rng(93).standard_normal(C * d)).astype(np.float32)
+    run_case(B, data, variant=variant, P=4, K=2, m=m, eta=0.05, R=2, J=20, kind="exp", mu=1.0, shift=0.0,
+             base=0, chunks=[7], use_ref=True)
+
+
 def test_softmax_growing_K_scaled_fourth_workload(B):
     """Shape of the AdaSync workload (P=8, m=128, eta=0.05, Delta=1, mu=2, K doubling 1 -> 8) on a
     smaller data set, with an interval short enough to cross every K within the run."""
