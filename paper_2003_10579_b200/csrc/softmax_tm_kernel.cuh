@@ -20,7 +20,7 @@
 //             (<= 31 shuffles for TG x 10 values) and a four-way sum in shared memory finish it.
 //   softmax   D = softmax(Z) - onehot(label), loss: 16 lanes per row.
 //   gradient  G += D^T X_tile: every thread, every row, own pairs, packed fp32x2 FMAs (the two
-//             features of a pair); D is stored duplicated so that no packing moves are needed.
+//             features of a pair); D is stored once and paired by register moves (see there).
 // Plain fp32 FMAs: at 20 FMA per 4-byte feature this path sits at the fp32 ridge, and the 1e-5
 // parity bound on the parameters rules out reduced-precision tensor-core operands.
 #pragma once
@@ -43,6 +43,7 @@ namespace ssim {
 
 constexpr int SMT_CP = 10;            // classes the layout is built for
 constexpr int SMT_WC = 2 * SMT_CP;    // tensor-memory columns per feature pair
+constexpr int SMT_DSTR = 12;          // floats per row of D in shared memory (10 classes, padded to whole 16-byte loads)
 constexpr int SMT_HEAD_BYTES = 4096;
 constexpr uint32_t SMT_TMEM_COLS = 256;
 
@@ -143,7 +144,7 @@ __global__ void __launch_bounds__(128 * NG) softmax_tm_kernel(NumericArgs a) {
 
   extern __shared__ __align__(128) unsigned char smem[];
   // head: barriers [2] @0 | tmem base @16 | first snapshot @20 | TileInfo [2] @32 | y [2][T] @96 | lossrow [T] @352
-  //       | misc [NW] @480 | delta [T][CP][2] @576 | red [NW][32] @3*1024
+  //       | misc [NW] @480 | delta [T][12] @576 | red [NW][32] @3*1024
   uint64_t* full = reinterpret_cast<uint64_t*>(smem);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 16);
   int* first_snap_s = reinterpret_cast<int*>(smem + 20);
@@ -367,7 +368,7 @@ __global__ void __launch_bounds__(128 * NG) softmax_tm_kernel(NumericArgs a) {
         if (is_max) dl = sc == label ? -sexcl * inv : inv;
         else dl = ez * inv - (sc == label ? 1.f : 0.f);
       }
-      if (sc < CP && sq < T) reinterpret_cast<float2*>(delta_s)[sq * CP + sc] = make_float2(dl, dl);
+      if (sc < SMT_DSTR && sq < T) delta_s[sq * SMT_DSTR + sc] = dl;
       loss_term = (sc == 0 && sq < ti.rows) ? zmax - zlab : 0.f;
       loss_s1 = (sc == 0 && sq < ti.rows) ? sexcl : 0.f;
     }
@@ -383,14 +384,23 @@ __global__ void __launch_bounds__(128 * NG) softmax_tm_kernel(NumericArgs a) {
         uint64_t x2[KP];
 #pragma unroll
         for (int k = 0; k < KP; ++k) x2[k] = xp[q * (DS / 2) + NT * k];
+        // D of the row: a shared-memory load delivers 4 bytes per lane and wavefront whatever its width, also when
+        // all lanes read the same address, so D is stored once (not as ready-made pairs) and paired by a register move
+        float dv[SMT_DSTR];
 #pragma unroll
-        for (int c2 = 0; c2 < CP / 2; ++c2) {
-          const ulonglong2 dd = reinterpret_cast<const ulonglong2*>(delta_s)[q * (CP / 2) + c2];
+        for (int c4 = 0; c4 < 2; ++c4) {
+          const float4 v = reinterpret_cast<const float4*>(delta_s)[q * (SMT_DSTR / 4) + c4];
+          dv[4 * c4] = v.x; dv[4 * c4 + 1] = v.y; dv[4 * c4 + 2] = v.z; dv[4 * c4 + 3] = v.w;
+        }
+        {
+          const float2 v = reinterpret_cast<const float2*>(delta_s)[q * (SMT_DSTR / 2) + 4];
+          dv[8] = v.x; dv[9] = v.y;
+        }
 #pragma unroll
-          for (int k = 0; k < KP; ++k) {
-            G[2 * c2][k] = ffma2(dd.x, x2[k], G[2 * c2][k]);
-            G[2 * c2 + 1][k] = ffma2(dd.y, x2[k], G[2 * c2 + 1][k]);
-          }
+        for (int c = 0; c < CP; ++c) {
+          const uint64_t dd = pack2(dv[c], dv[c]);
+#pragma unroll
+          for (int k = 0; k < KP; ++k) G[c][k] = ffma2(dd, x2[k], G[c][k]);
         }
       }
     }
