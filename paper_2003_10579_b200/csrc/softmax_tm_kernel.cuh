@@ -2,7 +2,7 @@
 // parameters live in TENSOR MEMORY, not in shared memory.
 //
 // One CTA of NT = 128 NG threads per replica, same producer / schedule walk as the other numeric
-// kernels (rows staged by bulk asynchronous copies, one tile of T = NG TG rows ahead).
+// kernels (rows staged by bulk asynchronous copies, a ring of tiles of T = NG TG rows).
 //
 // Ownership.  The d/2 pairs of adjacent features are dealt to the threads: thread t owns pairs
 // t + NT k (k < KP).  For its pairs and all classes it keeps the gradient accumulator G in registers
@@ -143,38 +143,41 @@ __global__ void __launch_bounds__(128 * NG) softmax_tm_kernel(NumericArgs a) {
   const long long my_j0 = a.run_j0 ? a.run_j0[r] : a.j0, my_iters = a.run_iters ? a.run_iters[r] : a.iters;
 
   extern __shared__ __align__(128) unsigned char smem[];
-  // head: barriers [2] @0 | tmem base @16 | first snapshot @20 | TileInfo [2] @32 | y [2][T] @96 | lossrow [T] @352
-  //       | misc [NW] @480 | delta [T][12] @576 | red [NW][32] @3*1024
+  // head (ring of S <= 4 tiles): barriers [4] @0 | tmem base @32 | first snapshot @36 | TileInfo [4] @48 | y [4][T] @160
+  //       | lossrow [T] @352 | misc [NW] @480 | delta [T][12] @576 | red [NW][32] @2048
+  const int S = a.stages;
   uint64_t* full = reinterpret_cast<uint64_t*>(smem);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 16);
-  int* first_snap_s = reinterpret_cast<int*>(smem + 20);
-  TmTileInfo* info_s = reinterpret_cast<TmTileInfo*>(smem + 32);
-  uint32_t* y_s = reinterpret_cast<uint32_t*>(smem + 96);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 32);
+  int* first_snap_s = reinterpret_cast<int*>(smem + 36);
+  TmTileInfo* info_s = reinterpret_cast<TmTileInfo*>(smem + 48);
+  uint32_t* y_s = reinterpret_cast<uint32_t*>(smem + 160);
   float* lossrow_s = reinterpret_cast<float*>(smem + 352);
   float* misc_s = reinterpret_cast<float*>(smem + 480);
   float* delta_s = reinterpret_cast<float*>(smem + 576);
   float* red_s = reinterpret_cast<float*>(smem + 2048);
-  static_assert(32 + 2 * sizeof(TmTileInfo) <= 96 && 96 + 8 * T <= 352 && 352 + 4 * T <= 480 && 480 + 4 * NW <= 576 &&
+  static_assert(48 + 4 * sizeof(TmTileInfo) <= 160 && 160 + 16 * T <= 352 && 352 + 4 * T <= 480 && 480 + 4 * NW <= 576 &&
                 576 + 8 * T * CP <= 2048 && 2048 + 128 * NW <= SMT_HEAD_BYTES, "head layout");
   float* rows_s = reinterpret_cast<float*>(smem + SMT_HEAD_BYTES);
-  uint32_t* pidx_s = reinterpret_cast<uint32_t*>(rows_s + (size_t)2 * T * DS);   // [m] sample rows of the producer's task
+  uint32_t* pidx_s = reinterpret_cast<uint32_t*>(rows_s + (size_t)S * T * DS);   // [m] sample rows of the producer's task
 
   if (tid == 0) {
-    for (int s = 0; s < 2; ++s) mbar_init(smem_addr(&full[s]), (uint32_t)T + 1u);
+    for (int s = 0; s < S; ++s) mbar_init(smem_addr(&full[s]), (uint32_t)T + 1u);
     mbar_fence_init();
   }
   if (warp == 1) tm_alloc(smem_addr(tmem_slot), SMT_TMEM_COLS);
   // The arithmetic reads whole row slots and whole tiles: features past d and rows past the end of a ragged tile
   // must hold finite numbers (they meet zero parameters / zero softmax terms), so the slots start as zeros.
-  for (int i = tid; i < 2 * T * DS / 4; i += NT) reinterpret_cast<float4*>(rows_s)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int i = tid; i < S * T * DS / 4; i += NT) reinterpret_cast<float4*>(rows_s)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   __syncthreads();
 
   ScheduleWalk walk;
   walk.done = true;
-  auto issue_tile = [&](long long tile_no) {
+  int prod_st = 0;      // tiles are issued in order: the producer's stage is a counter
+  auto issue_tile = [&]() {
     if (walk.done) return;
-    const int st = (int)(tile_no & 1);
+    const int st = prod_st;
+    if (++prod_st == S) prod_st = 0;
     const uint32_t bar = smem_addr(&full[st]);
     const int rows = min(T, m - walk.k * T);
     if (walk.k == 0) {   // a new task: its m sample rows are drawn once, 32 at a time (only this warp uses the table)
@@ -214,7 +217,7 @@ __global__ void __launch_bounds__(128 * NG) softmax_tm_kernel(NumericArgs a) {
     walk.start(a, r, my_j0, my_iters);
     walk.tiles_per_task = (m + T - 1) / T;
     if (lane == 0) *first_snap_s = walk.done ? 0 : (int)walk.cur.snap;
-    for (int s = 0; s < 2; ++s) issue_tile(s);
+    for (int s = 0; s < S; ++s) issue_tile();
   }
   tm_fence_before();
   __syncthreads();
@@ -260,9 +263,9 @@ __global__ void __launch_bounds__(128 * NG) softmax_tm_kernel(NumericArgs a) {
   const int sq = st_tid >> 4, sc = st_tid & 15;    // 16 lanes per row
   const int red_idx = tm_reduce_index<NV>(lane);
 
-  for (long long it = 0; my_iters > 0; ++it) {
-    const int st = (int)(it & 1);
-    const uint32_t parity = (uint32_t)((it >> 1) & 1);
+  int st = 0;                // stage and phase parity of tile `it`, as counters
+  uint32_t parity = 0;
+  for (long long it = 0; my_iters > 0; ++it, parity ^= (uint32_t)(st + 1 == S), st = (st + 1 == S ? 0 : st + 1)) {
     const bool ok = mbar_wait(smem_addr(&full[st]), parity);
     const TmTileInfo ti = info_s[st];
     const float* tile = rows_s + (size_t)st * T * DS;
@@ -333,7 +336,7 @@ __global__ void __launch_bounds__(128 * NG) softmax_tm_kernel(NumericArgs a) {
     tm_fence_before();
     if (__syncthreads_or(!ok)) { failed = true; break; }   // (A) partial logits published; everyone is past the previous tile
     tm_fence_after();
-    if (warp == 0 && it >= 1) issue_tile(it + 1);          // into the stage of tile it - 1
+    if (warp == 0 && it >= 1) issue_tile();                // tile it + S - 1, into the stage of tile it - 1
 
     // ---- softmax stage: thread (sq, sc) owns logit (row sq, class sc) ----
     float loss_term = 0.f, loss_s1 = 0.f;
@@ -488,9 +491,9 @@ __global__ void __launch_bounds__(128 * NG) softmax_tm_kernel(NumericArgs a) {
   if (warp == 1) tm_dealloc(tmem, SMT_TMEM_COLS);
 }
 
-inline size_t softmax_tm_smem_bytes(int T, int d, int m) {
+inline size_t softmax_tm_smem_bytes(int S, int T, int d, int m) {
   const int nt = 128 * SMX_TM_NG, kp = (d / 2 + nt - 1) / nt;
-  const size_t need = (size_t)SMT_HEAD_BYTES + (size_t)2 * T * (2 * nt * kp) * 4 + (size_t)m * 4;
+  const size_t need = (size_t)SMT_HEAD_BYTES + (size_t)S * T * (2 * nt * kp) * 4 + (size_t)m * 4;
   // one CTA per SM, whatever the shape: two CTAs' tensor-memory allocations would still fit, a third would wait
   return need < (size_t)(116 << 10) ? (size_t)(116 << 10) : need;
 }
@@ -499,17 +502,19 @@ inline size_t softmax_tm_smem_bytes(int T, int d, int m) {
 inline bool softmax_tm_supported(int d, int C, int m) {
   constexpr int NT = 128 * SMX_TM_NG, T = SMX_TM_NG * SMX_TM_TG;
   const int kp = (d / 2 + NT - 1) / NT;
-  return C <= SMT_CP && kp * SMX_TM_NG * SMT_WC <= (int)SMT_TMEM_COLS && softmax_tm_smem_bytes(T, d, m) <= (size_t)(226 << 10);
+  return C <= SMT_CP && kp * SMX_TM_NG * SMT_WC <= (int)SMT_TMEM_COLS && softmax_tm_smem_bytes(2, T, d, m) <= (size_t)(226 << 10);
 }
 
 template <int KP>
 cudaError_t launch_softmax_tm(NumericArgs& a, cudaStream_t stream) {
   constexpr int NG = SMX_TM_NG, TG = SMX_TM_TG;
   auto kern = a.is_async ? softmax_tm_kernel<NG, KP, TG, true> : softmax_tm_kernel<NG, KP, TG, false>;
-  const size_t smem = softmax_tm_smem_bytes(NG * TG, a.d, a.m);
+  int S = 4;   // tiles in the ring: as many as shared memory holds, two at least
+  while (S > 2 && softmax_tm_smem_bytes(S, NG * TG, a.d, a.m) > (size_t)(226 << 10)) --S;
+  const size_t smem = softmax_tm_smem_bytes(S, NG * TG, a.d, a.m);
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  a.stages = 2;
+  a.stages = S;
   kern<<<a.R, 128 * NG, smem, stream>>>(a);
   return cudaGetLastError();
 }
