@@ -89,7 +89,8 @@ typedef struct {
  * (Eq. 2 / Eq. 3: w_{j+1} = w_j - (eta/K) sum_l g(w_tau(l,j), xi_l,j)), minibatch size m per
  * worker, drawn with replacement from all n samples.  Initial parameters are zero until
  * sim_set_params.  problem may be NULL or have model SIM_NONE for a clock-only simulation.
- * Errors: SIM_ERR_ARG for P not in [1, SIM_MAX_P], K not in [1, P], m < 1, n_replicas < 1,
+ * Errors: SIM_ERR_ARG for P not in [1, SIM_MAX_P], K not in [1, P], m < 1, m > 2^26, an m whose
+ * index table does not fit in shared memory beside two tiles of rows of this d, n_replicas < 1,
  * mu <= 0 or NaN, shift < 0 or not finite, d % 4 != 0, misaligned or NULL X, missing y / label,
  * replica ids beyond 2^32; SIM_ERR_ALLOC / SIM_ERR_CUDA otherwise.  *out is NULL on failure.
  */
@@ -235,8 +236,11 @@ sim_status sim_sweep_host(const sim_problem* problem, int32_t P, int32_t n_runs,
  * (SIM_NOALLOC_SCRATCH_BYTES of device memory on every GPU that loads the library, held until the
  * process exits), which bounds the problem: P <= SIM_NOALLOC_MAX_P, n_replicas <= SIM_NOALLOC_MAX_REPLICAS and
  * n_replicas * P <= SIM_NOALLOC_MAX_REPLICA_WORKERS; larger requests return SIM_ERR_ARG and launch
- * nothing.  The first call on each device looks up the array's device address; make that first
- * call outside any stream capture.  All calls on a device share the array and each call clears
+ * nothing.  The first call on each device looks up the array's device address and, with CUDA's lazy
+ * module loading, is also the moment the driver loads the library's device code and the array itself
+ * onto that device (which takes device memory and can fail if none is left): make that first call at
+ * start-up, outside any stream capture and before the memory is claimed by others; the promise of
+ * no allocation holds for every later call.  All calls on a device share the array and each call clears
  * the part it uses before it starts, so two calls whose GPU work overlaps (different streams or
  * threads) race: serialise them.  Work is enqueued on `cuda_stream`; the call does not wait for
  * it.  On failure sim_noalloc_last_error() describes the cause (per host thread).

@@ -235,6 +235,14 @@ def schedule_noalloc(out, *, P, K, variant, delay_kind, mu, shift=0.0, seed, n_r
     Simulation.trace) because the library may not create them.  For callers that cannot call
     cudaMalloc; the worker state sits in a fixed array inside the library, so sizes are capped and
     calls on one device must not overlap."""
+    Ks = P if t_interval > 0 else K
+    need = {"t": (torch.float64, n_replicas * iters), "K": (_U16, n_replicas * iters),
+            "worker": (_U16, n_replicas * iters * Ks), "stale": (_U32, n_replicas * iters * Ks),
+            "seq": (_U32, n_replicas * iters * Ks)}
+    for k, (dt, count) in need.items():     # the library writes through raw pointers: a wrong buffer would be an out-of-bounds write
+        t = out[k]
+        if not (t.is_cuda and t.is_contiguous() and t.dtype == dt and t.numel() >= count):
+            raise ValueError("schedule_noalloc: out[%r] must be a contiguous CUDA tensor of %s with at least %d elements" % (k, dt, count))
     st = lib.sim_schedule_noalloc(P, K, VARIANTS[variant], SimDelay(DELAYS[delay_kind], mu, shift), seed,
                                   replica_base, n_replicas, K0, t_interval, iters,
                                   *[_ptr(out[k]) for k in ("t", "K", "worker", "stale", "seq")],

@@ -37,6 +37,11 @@ struct MlpScratch {
   float* db1_part = nullptr;       // [R][Kmax][m/32][H]       column sums of delta1 per 32-row group
   float* loss_part = nullptr;      // [R][Kmax][m/32]
   int* rows_tab = nullptr;         // [R][Kmax][m]             sample row of every minibatch draw of the current update
+  // |w_{j+1} - w_ref|^2 of the current update, in pieces: one partial per (W1 tile, epilogue group) from the dW1 kernel,
+  // one per 32 hidden units ([b1 | W2 | b2] part) from the head kernel; the last piece to arrive adds them in index order
+  float* dist_w1 = nullptr;        // [R][(d/128) (H/Hn) 2]
+  float* dist_head = nullptr;      // [R][H/32]
+  int* dist_cnt = nullptr;         // [R] W1 pieces that have arrived
   int H = 0, C = 0, d = 0, m = 0, Kmax = 0, n_slots = 0, R = 0;
   long long n = 0;
 };
@@ -101,6 +106,7 @@ __global__ void mlp_rows_kernel(MlpArgs g) {
   const MlpScratch& sc = g.sc;
   const int l = blockIdx.x % sc.Kmax, r = blockIdx.x / sc.Kmax;
   const int K = (int)a.K_used[(size_t)r * a.cap + g.j];
+  if (l == 0 && threadIdx.x == 0) sc.dist_cnt[r] = 0;
   if (l >= K) return;
   const size_t ent = ((size_t)r * a.cap + g.j) * a.K_stride + l;
   const uint32_t worker = a.worker[ent], seq = a.seq[ent];
@@ -170,6 +176,10 @@ __global__ void __launch_bounds__(MLP_HEAD_THREADS, 3) mlp_head_kernel(MlpArgs g
   const float scale = (float)((double)a.eta / ((double)K * (double)m));
   const float* wc = a.pool + ((size_t)r * a.n_slots + cur) * a.slot_stride + dH;      // [b1 | W2 | b2] of w_j
   float* wn = a.pool + ((size_t)r * a.n_slots + fresh) * a.slot_stride + dH;
+  // with a reference vector: this CTA's share of |w_{j+1} - w_ref|^2 (its entries of b1, W2, b2), summed in a fixed order
+  const float* wref = a.w_ref ? a.w_ref + dH : nullptr;
+  float dd = 0.f;
+  auto dist_term = [&](size_t p, float w_new) { if (wref) { const float e = w_new - wref[p]; dd = fmaf(e, e, dd); } };
   // W2 rows cb*32 .. cb*32+31: 32 x C consecutive parameters
   for (int e = tid; e < 32 * C; e += MLP_HEAD_THREADS) {
     const int col = e / C, c = e % C;
@@ -177,13 +187,17 @@ __global__ void __launch_bounds__(MLP_HEAD_THREADS, 3) mlp_head_kernel(MlpArgs g
 #pragma unroll
     for (int w = 0; w < 8; ++w) gsum += d2_s[w][col][c];
     const size_t p = (size_t)H + (size_t)(cb * 32) * C + e;
-    wn[p] = fmaf(-scale, gsum, wc[p]);
+    const float w_new = fmaf(-scale, gsum, wc[p]);
+    wn[p] = w_new;
+    dist_term(p, w_new);
   }
   if (tid < 32) {                                             // b1: partial column sums of delta1 written by the forward kernel
     const int col = cb * 32 + tid, parts = m / 32;
     float gsum = 0.f;
     for (int q = 0; q < K * parts; ++q) gsum += sc.db1_part[((size_t)r * sc.Kmax * parts + q) * H + col];
-    wn[col] = fmaf(-scale, gsum, wc[col]);
+    const float w_new = fmaf(-scale, gsum, wc[col]);
+    wn[col] = w_new;
+    dist_term((size_t)col, w_new);
   }
   if (cb == 0 && warp == 1) {
     if (lane < C) {
@@ -191,14 +205,28 @@ __global__ void __launch_bounds__(MLP_HEAD_THREADS, 3) mlp_head_kernel(MlpArgs g
 #pragma unroll
       for (int w = 0; w < 8; ++w) gsum += b2_s[w][lane];
       const size_t p = (size_t)H + (size_t)H * C + lane;
-      wn[p] = fmaf(-scale, gsum, wc[p]);
+      const float w_new = fmaf(-scale, gsum, wc[p]);
+      wn[p] = w_new;
+      dist_term(p, w_new);
     }
     if (lane == 31) {
       const int parts = m / 32;
       float ls = 0.f;
       for (int q = 0; q < K * parts; ++q) ls += sc.loss_part[(size_t)r * sc.Kmax * parts + q];
       a.loss[(size_t)r * a.cap + j] = ls / ((float)K * (float)m);
-      a.dist2[(size_t)r * a.cap + j] = 0.f;
+      if (!wref) a.dist2[(size_t)r * a.cap + j] = 0.f;      // otherwise the dW1 kernel records it once W1 is updated
+    }
+  }
+  if (wref) {
+    __shared__ float dist_s[8];
+    dd = warp_sum(dd);
+    if (lane == 0) dist_s[warp] = dd;
+    __syncthreads();
+    if (tid == 0) {
+      float tot = 0.f;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) tot += dist_s[w];
+      sc.dist_head[(size_t)r * ncb + cb] = tot;
     }
   }
 }
@@ -206,7 +234,7 @@ __global__ void __launch_bounds__(MLP_HEAD_THREADS, 3) mlp_head_kernel(MlpArgs g
 // ---- host side -----------------------------------------------------------------------------------
 inline void mlp_scratch_free(MlpScratch& s) {
   cudaFree(s.rows_tab); cudaFree(s.Xq); cudaFree(s.W1qT); cudaFree(s.D1q); cudaFree(s.Hact); cudaFree(s.D2);
-  cudaFree(s.db1_part); cudaFree(s.loss_part);
+  cudaFree(s.db1_part); cudaFree(s.loss_part); cudaFree(s.dist_w1); cudaFree(s.dist_head); cudaFree(s.dist_cnt);
   s = MlpScratch{};
 }
 
@@ -226,6 +254,9 @@ inline cudaError_t mlp_scratch_alloc(MlpScratch& s, const float* X, long long n,
   MLP_ALLOC(s.db1_part, tasks * (m / 32) * H)
   MLP_ALLOC(s.loss_part, tasks * (m / 32))
   MLP_ALLOC(s.rows_tab, tasks * m)
+  MLP_ALLOC(s.dist_w1, (size_t)R * (d / 128) * (H / 64) * 2)      // at most H/64 column parts per 128-row slab
+  MLP_ALLOC(s.dist_head, (size_t)R * (H / 32))
+  MLP_ALLOC(s.dist_cnt, (size_t)R)
 #undef MLP_ALLOC
   to_bf16_kernel<<<1184, 256, 0, stream>>>(X, s.Xq, (long long)n * d);
   return cudaGetLastError();

@@ -419,7 +419,7 @@ inline __host__ __device__ int tc_dw1_cols(int H) {
     if (H % p == 0 && H / p <= 256 && (H / p) % 64 == 0) return H / p;
   return 64;
 }
-struct TcDw1Layout { int stages, stage_bytes, wslots, off_w, off_q, off_bars, off_tmem, off_fail, total; };
+struct TcDw1Layout { int stages, stage_bytes, wslots, off_w, off_q, off_bars, off_tmem, off_fail, off_dist, total; };
 inline __host__ __device__ TcDw1Layout tc_dw1_layout(int H) {
   TcDw1Layout L;
   const int budget = 224 << 10;
@@ -433,7 +433,8 @@ inline __host__ __device__ TcDw1Layout tc_dw1_layout(int H) {
   L.off_bars = L.off_q + 2 * DW1_QSTAGE;
   L.off_tmem = L.off_bars + 8 * (2 * L.stages + 4 + 2 * L.wslots);
   L.off_fail = L.off_tmem + 16;
-  L.total = L.off_fail + 16 + 1024;
+  L.off_dist = L.off_fail + 16;        // [2 groups][4 warps] partial distances
+  L.total = L.off_dist + 32 + 1024;
   return L;
 }
 
@@ -475,6 +476,7 @@ mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
   const uint32_t bars = base_addr + L.off_bars;     // full[S] | empty[S] | acc_full[2] | acc_empty[2] | wfull[NB] | wempty[NB]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base + L.off_tmem);
   volatile int* fail_s = reinterpret_cast<volatile int*>(base + L.off_fail);     // one flag per epilogue group
+  float* dist_s = reinterpret_cast<float*>(base + L.off_dist);
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (S + s); };
   auto acc_full = [&](int b) { return bars + 8u * (2 * S + b); };
@@ -602,8 +604,16 @@ mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
       float* wn = a.pool + ((size_t)r * a.n_slots + fresh) * a.slot_stride + (((size_t)slab * (H >> 5) + ((part * Hn) >> 5)) << 12);
       __nv_bfloat16* wq = sc.W1qT + ((size_t)r * sc.n_slots + fresh) * dH + ((size_t)(2 * slab) * H + part * Hn) * 64;
       const uint32_t trow = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * Hn);
+      // reference parameters of this thread's row (row-major [d][H], as the caller gave them) for |w_{j+1} - w_ref|^2
+      const float4* wref_row = a.w_ref ? reinterpret_cast<const float4*>(a.w_ref + (size_t)(slab * 128 + rloc) * H + part * Hn) : nullptr;
+      float dd = 0.f;
       for (int b = grp; b < nb; b += 2, wp.step(NB, 2)) {
         const int s = wp.s;
+        float4 wr[8];                                   // requested before the waits below, so that their latency hides there
+        if (wref_row) {
+#pragma unroll
+          for (int i4 = 0; i4 < 8; ++i4) wr[i4] = wref_row[b * 8 + i4];
+        }
         bool ok = mbar_wait(wfull(s), wp.ph);
         if (ok && b == grp) ok = mbar_wait(acc_full(buf), (uint32_t)((i >> 1) & 1));
         if (!ok) fail_s[grp] = 1;
@@ -625,6 +635,10 @@ mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
           qrow[(4 * i4 + 1) * 64] = __float2bfloat16_rn(w.y);
           qrow[(4 * i4 + 2) * 64] = __float2bfloat16_rn(w.z);
           qrow[(4 * i4 + 3) * 64] = __float2bfloat16_rn(w.w);
+          if (wref_row) {
+            const float e0 = w.x - wr[i4].x, e1 = w.y - wr[i4].y, e2 = w.z - wr[i4].z, e3 = w.w - wr[i4].w;
+            dd = fmaf(e0, e0, dd); dd = fmaf(e1, e1, dd); dd = fmaf(e2, e2, dd); dd = fmaf(e3, e3, dd);
+          }
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         group_barrier(1 + grp, 128);
@@ -641,6 +655,27 @@ mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
       tc_fence_before();                 // this warp's reads of the buffer are done: hand it back
       __syncwarp();
       if (lane == 0) mbar_arrive(acc_empty(buf));
+      if (wref_row) {
+        // This group's share of the tile goes to its own entry; the group that delivers a replica's last entry
+        // adds all of them, and the head kernel's, in index order and records the distance (fixed order of sums).
+        dd = warp_sum(dd);
+        if (lane == 0) dist_s[grp * 4 + q] = dd;
+        group_barrier(1 + grp, 128);
+        if (leader) {
+          const int per_r = slabs * parts * 2;
+          float* mine = sc.dist_w1 + (size_t)r * per_r;
+          mine[(slab * parts + part) * 2 + grp] = (dist_s[grp * 4] + dist_s[grp * 4 + 1]) + (dist_s[grp * 4 + 2] + dist_s[grp * 4 + 3]);
+          __threadfence();
+          if (atomicAdd(sc.dist_cnt + r, 1) == per_r - 1) {
+            __threadfence();
+            float tot = 0.f;
+            for (int i2 = 0; i2 < per_r; ++i2) tot += __ldcg(mine + i2);
+            for (int i2 = 0; i2 < H / 32; ++i2) tot += __ldcg(sc.dist_head + (size_t)r * (H / 32) + i2);
+            a.dist2[(size_t)r * a.cap + j] = tot;
+          }
+        }
+        group_barrier(1 + grp, 128);     // dist_s may be overwritten by the next tile
+      }
     }
     if (leader) bulk_wait_all();
   } else {

@@ -230,7 +230,8 @@ sim_status launch_linear1(sim_handle* h, NumericArgs& a) {
   if (S > 8) S = 8;
   size_t smem = linear1_smem_bytes(NT, T, S, d, a.m);
   while (smem > (size_t)(226 << 10) && S > 2) { --S; smem = linear1_smem_bytes(NT, T, S, d, a.m); }
-  if (smem > (size_t)(226 << 10)) return fail(h, SIM_ERR_ARG, "d too large for the row staging buffers");
+  if (smem > (size_t)(226 << 10))
+    return fail(h, SIM_ERR_ARG, "the row staging buffers (d) and the minibatch index table (m) do not fit in shared memory with this tuning");
   a.stages = S;
   auto kern = a.is_async ? linear1_kernel<NT, CHUNKS, T, true> : linear1_kernel<NT, CHUNKS, T, false>;
   CUDA_TRY(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -257,6 +258,20 @@ sim_status run_linear1(sim_handle* h, NumericArgs& a) {
   }
   if (d4 <= 2048) return launch_linear1<512, 4, 2>(h, a);
   return fail(h, SIM_ERR_ARG, "d > 8192 is not supported by the linear-model kernel");
+}
+
+// Shared memory the linear-model kernel needs at its smallest ring (two stages) with the tile shape the
+// dispatch above picks for d when no tuning is set: rows of the ring plus the m-entry index table.
+size_t linear1_min_smem(int d, int m, int R) {
+  const int d4 = d / 4;
+  int NT = 512, T = 2;
+  if (d4 <= 32) { NT = 32; T = 8; }
+  else if (d4 <= 64) { NT = 64; T = 8; }
+  else if (d4 <= 128) { NT = 128; T = 4; }
+  else if (d4 <= 256) { NT = 128; T = 4; }
+  else if (d4 <= 512) { NT = 256; T = 4; }
+  else if (d4 <= 1024) { NT = 256; T = R > 148 ? 2 : 4; }
+  return linear1_smem_bytes(NT, T, 2, d, m);
 }
 
 sim_status device_error(const sim_handle* h) {
@@ -322,6 +337,8 @@ sim_status sim_create(const sim_problem* problem, int32_t P, int32_t K, sim_vari
   if (K < 1 || K > P) return fail(nullptr, SIM_ERR_ARG, "K must be in [1, P]");
   if ((int)variant < 0 || (int)variant > 3) return fail(nullptr, SIM_ERR_ARG, "unknown variant");
   if (m < 1) return fail(nullptr, SIM_ERR_ARG, "m must be >= 1");
+  // the index stream packs draw q as chunk q / 4 into 24 bits of the counter
+  if (m > (1 << 26)) return fail(nullptr, SIM_ERR_ARG, "m must be at most 2^26 (the minibatch index stream has 2^24 chunks of four draws)");
   if (n_replicas < 1) return fail(nullptr, SIM_ERR_ARG, "n_replicas must be >= 1");
   if (replica_base < 0 || replica_base + (int64_t)n_replicas > (int64_t)1 << 32)
     return fail(nullptr, SIM_ERR_ARG, "global replica ids must fit in 32 bits");
@@ -353,6 +370,9 @@ sim_status sim_create(const sim_problem* problem, int32_t P, int32_t K, sim_vari
     }
     if ((prob.model == SIM_LSQ || prob.model == SIM_LOGISTIC) && prob.d > 8192)
       return fail(nullptr, SIM_ERR_ARG, "d > 8192 is not supported by the linear-model kernel");
+    if ((prob.model == SIM_LSQ || prob.model == SIM_LOGISTIC) && linear1_min_smem(prob.d, m, n_replicas) > (size_t)(226 << 10))
+      return fail(nullptr, SIM_ERR_ARG, "m is too large for this d: the kernel keeps two tiles of sample rows and an m-entry index table "
+                                        "(4 m bytes) in shared memory");
   }
 
   sim_handle* h = new (std::nothrow) sim_handle();
@@ -417,7 +437,9 @@ sim_status sim_set_adasync(sim_handle* h, int32_t K0, double t_interval) {
     if (K0 < 1 || K0 > h->P) return fail(h, SIM_ERR_ARG, "K0 must be in [1, P]");
     h->K0 = K0; h->t_interval = t_interval; h->K_stride = h->P; h->ada_loss = false;
   } else {
-    h->K0 = 0; h->t_interval = 0.0; h->K_stride = h->K;
+    // switching the schedule off also switches off the loss-driven rule: with no interval there is nothing to
+    // pause at, and the trace rows go back to K entries
+    h->K0 = 0; h->t_interval = 0.0; h->K_stride = h->K; h->ada_loss = false; h->F0_ready = false;
   }
   return SIM_OK;
 }
@@ -458,7 +480,7 @@ sim_status sim_run(sim_handle* h, int64_t iters) {
   // Loss-driven K: replicas pause where an update starts in a new interval and K may still grow; each
   // round schedules every replica up to its next pause (or the target), runs the arithmetic that far,
   // evaluates the full-data risk and sets the paused replicas' new K.  Rounds = interval crossings + 1.
-  const bool adaptive = h->ada_loss;
+  const bool adaptive = h->ada_loss && h->t_interval > 0.0;
   if (adaptive) {
     if (!h->F0_ready) { if ((st = eval_into(h, h->F0)) != SIM_OK) return st; h->F0_ready = true; }
     sa.adaptive = 1; sa.target = h->n_updates + iters; sa.done = h->done; sa.run_j0 = h->run_j0; sa.run_iters = h->run_iters;

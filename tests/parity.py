@@ -51,10 +51,34 @@ def rel_norm(a, b):
     return np.linalg.norm(a - b) / (nb if nb > 0 else 1.0)
 
 
+def max_elem_err(w_gpu, w_ora):
+    """Largest element-wise difference relative to the largest parameter: max_i |dw_i| / max_i |w_i|."""
+    a, b = np.asarray(w_gpu, np.float64), np.asarray(w_ora, np.float64)
+    top = np.abs(b).max()
+    return np.abs(a - b).max() / (top if top > 0 else 1.0)
+
+
 def assert_params_close(w_gpu, w_ora, what="", rtol=PARAM_RTOL):
+    """Two bounds at the same tolerance: the relative 2-norm of the difference, and every single element against
+    the largest parameter (a norm alone would let one element of thousands be off by much more).  Returns the
+    larger of the two measures."""
     e = rel_norm(w_gpu, w_ora)
     assert e <= rtol, "%s: |w_gpu - w_oracle| / |w_oracle| = %.3g > %.1g" % (what, e, rtol)
-    return e
+    a, b = np.asarray(w_gpu, np.float64), np.asarray(w_ora, np.float64)
+    m = max_elem_err(a, b)
+    if m > rtol:
+        i = int(np.argmax(np.abs(a - b)))
+        raise AssertionError("%s: element %d differs by %.3g (gpu %.9g oracle %.9g), %.3g of the largest parameter > %.1g" % (
+            what, i, abs(a.flat[i] - b.flat[i]), a.flat[i], b.flat[i], m, rtol))
+    return max(e, m)
+
+
+def strict_loss_stats(l_gpu, l_ora, rtol=LOSS_RTOL):
+    """The plain relative bound, with no allowance for trajectory drift: (fraction of updates inside rtol, worst
+    relative error), relative to max(|L_oracle|, 1e-6 L_0)."""
+    l_gpu, l_ora = np.asarray(l_gpu, np.float64), np.asarray(l_ora, np.float64)
+    rel = np.abs(l_gpu - l_ora) / np.maximum(np.abs(l_ora), 1e-6 * abs(l_ora.flat[0]))
+    return float((rel <= rtol).mean()), float(rel.max())
 
 
 def assert_loss_close(l_gpu, l_ora, what="", rtol=LOSS_RTOL, gnorm=None, dw=0.0):

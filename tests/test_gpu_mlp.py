@@ -24,14 +24,15 @@ def B():
 
 
 def run_mlp_case(B, data, w0, *, variant, P, K, m, eta, R, J, kind="exp", mu=1.0, shift=0.0, seed=3, base=0, K0=0,
-                 ti=0.0, replicas=None, chunks=(1, 1)):
+                 ti=0.0, replicas=None, chunks=(1, 1), w_ref=None):
     dev = to_device(data)
     sim = B.Simulation(dev, P=P, K=K, variant=variant, delay_kind=kind, mu=mu, shift=shift, eta=eta, m=m,
-                       seed=seed, n_replicas=R, replica_base=base)
+                       seed=seed, n_replicas=R, replica_base=base, w_ref=None if w_ref is None else torch.from_numpy(w_ref).cuda())
     if ti > 0:
         sim.set_adasync(K0, ti)
     sim.set_params(torch.from_numpy(w0).cuda())
-    kw = dict(P=P, K=K, variant=variant, delay_kind=kind, mu=mu, shift=shift, eta=eta, m=m, seed=seed, K0=K0, t_interval=ti)
+    kw = dict(P=P, K=K, variant=variant, delay_kind=kind, mu=mu, shift=shift, eta=eta, m=m, seed=seed, K0=K0, t_interval=ti,
+              w_ref=w_ref)
     replicas = list(range(R)) if replicas is None else replicas
     oras = {r: oracle_replica(data, w0, base + r, **kw) for r in replicas}
     plan = list(chunks) + ([J - sum(chunks)] if J > sum(chunks) else [])
@@ -50,10 +51,17 @@ def run_mlp_case(B, data, w0, *, variant, P, K, m, eta, R, J, kind="exp", mu=1.0
     assert_schedule_equal(tr, sched)
     worst_l = 0.0
     for r, o in oras.items():
-        ol = o.trace_arrays(K_stride=tr["worker"].shape[2])["loss"].astype(np.float64)
+        ot = o.trace_arrays(K_stride=tr["worker"].shape[2])
+        ol = ot["loss"].astype(np.float64)
         err = np.abs(tr["loss"][r] - ol) / np.abs(ol)
         assert err.max() <= MLP_LOSS_RTOL, "%s replica %d: loss err %.3g at update %d" % (variant, r, err.max(), err.argmax())
         worst_l = max(worst_l, err.max())
+        if w_ref is None:
+            assert not tr["dist2"][r].any()
+        else:       # Section 2.3's distance to a reference point, |w_{j+1} - w_ref|^2, over all four parameter blocks
+            od = ot["dist2"].astype(np.float64)
+            derr = np.abs(tr["dist2"][r] - od) / od
+            assert derr.max() <= MLP_LOSS_RTOL, "%s replica %d: dist2 err %.3g at update %d" % (variant, r, derr.max(), derr.argmax())
     print("mlp %s K=%d d=%d H=%d: worst param err %.2e, worst loss err %.2e, final loss %.4f" % (
         variant, K, data["X"].shape[1], data["hidden"], worst_w, worst_l, tr["loss"][replicas[0], -1]))
     return tr
@@ -64,7 +72,10 @@ def run_mlp_case(B, data, w0, *, variant, P, K, m, eta, R, J, kind="exp", mu=1.0
 def test_mlp_variants_and_shapes(B, variant, d, H, C, m, K, P):
     data = inputs.make_mixture(4096, d, C, 0.5 if d < 1000 else 0.1, 95, "mlp2", H)
     w0 = inputs.mlp_init(d, H, C, 96)
-    run_mlp_case(B, data, w0, variant=variant, P=P, K=K, m=m, eta=0.02, R=3, J=12 if d > 1000 else 25, base=1)
+    # every other case carries a reference vector: another draw of the initial weights, shifted so that no block of the
+    # parameter vector is close to it by accident
+    w_ref = (inputs.mlp_init(d, H, C, 197) + np.float32(0.01)) if (d + K) % 2 == 0 or variant == "kbatchasync" else None
+    run_mlp_case(B, data, w0, variant=variant, P=P, K=K, m=m, eta=0.02, R=3, J=12 if d > 1000 else 25, base=1, w_ref=w_ref)
 
 
 @pytest.mark.parametrize("variant", ["kasync", "kbatchasync"])

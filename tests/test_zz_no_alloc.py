@@ -56,8 +56,18 @@ def test_no_alloc_entry_point_matches_regular_path_twice_in_a_row():
 def test_no_alloc_entry_point_refuses_what_the_fixed_array_cannot_hold():
     from paper_2003_10579_b200 import binding as B
     kw = dict(P=32, K=1, variant="ksync", delay_kind="exp", mu=1.0, seed=0)
-    out = {k: torch.zeros(8, dtype=torch.float64, device="cuda") for k in ("t", "K", "worker", "stale", "seq")}
+    types = {"t": torch.float64, "K": _U16, "worker": _U16, "stale": _U32, "seq": _U32}
+    out = {k: torch.zeros(4097, dtype=torch.int64, device="cuda").to(dt) for k, dt in types.items()}
     for R in (4097, 2049):          # too many replicas; too many replica x worker pairs
         with pytest.raises(B.SimError) as e:
             B.schedule_noalloc(out, n_replicas=R, iters=1, **kw)
         assert e.value.status == 1 and "SIM_NOALLOC_MAX" in str(e.value)
+
+
+def test_no_alloc_binding_refuses_buffers_the_library_would_overrun():
+    from paper_2003_10579_b200 import binding as B
+    kw = dict(P=4, K=2, variant="ksync", delay_kind="exp", mu=1.0, seed=0)
+    types = {"t": torch.float64, "K": _U16, "worker": _U16, "stale": _U32, "seq": _U32}
+    out = {k: torch.zeros(16, dtype=torch.int64, device="cuda").to(dt) for k, dt in types.items()}
+    with pytest.raises(ValueError):          # worker / stale / seq need 4 x 4 x 2 = 32 entries
+        B.schedule_noalloc(out, n_replicas=4, iters=4, **kw)
