@@ -173,6 +173,16 @@ sim_status sim_eval_loss(sim_handle* h, float* loss);
  */
 sim_status sim_error_curve(const sim_handle* h, const double* grid, int32_t n_grid, float* mean_loss, int32_t* count);
 
+/*
+ * Diagnostic (no counterpart in the paper): exercises the path by which a device-side wait that runs out is
+ * reported.  Every wait in the library's kernels is bounded; when one gives up, the block votes, sets the handle's
+ * error word and drains, and the next synchronising call returns SIM_ERR_TIMEOUT and leaves the handle unusable.
+ * This call enqueues a one-block kernel that waits about a thousand polls on a barrier nobody arrives at, so that
+ * exactly this happens: sim_trace_size / sim_get_* then return SIM_ERR_TIMEOUT and sim_run SIM_ERR_STATE.  The
+ * kernel ends by itself; the device and other handles are unaffected.  Returns SIM_OK after enqueueing.
+ */
+sim_status sim_selftest_wait_timeout(sim_handle* h);
+
 /* Number of parameters of the handle's model (0 for SIM_NONE). */
 int64_t sim_n_params(const sim_handle* h);
 

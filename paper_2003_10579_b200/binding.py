@@ -20,7 +20,7 @@ STATUS = {0: "SIM_OK", 1: "SIM_ERR_ARG", 2: "SIM_ERR_ALLOC", 3: "SIM_ERR_CUDA", 
           5: "SIM_ERR_STATE", 6: "SIM_ERR_INTERNAL"}
 
 EXPORTS = ["sim_create", "sim_set_params", "sim_set_adasync", "sim_set_adasync_loss", "sim_set_tuning", "sim_reserve", "sim_run",
-           "sim_trace_size", "sim_get_trace", "sim_get_params", "sim_eval_loss", "sim_error_curve", "sim_n_params", "sim_last_error",
+           "sim_trace_size", "sim_get_trace", "sim_get_params", "sim_eval_loss", "sim_error_curve", "sim_selftest_wait_timeout", "sim_n_params", "sim_last_error",
            "sim_destroy", "sim_draw_delays", "sim_draw_indices", "sim_simulate_host", "sim_sweep_host", "sim_schedule_noalloc",
            "sim_noalloc_last_error"]
 
@@ -60,6 +60,7 @@ def _load():
     L.sim_get_params.argtypes = [vp, vp]
     L.sim_eval_loss.argtypes = [vp, vp]
     L.sim_error_curve.argtypes = [vp, vp, i32, vp, vp]
+    L.sim_selftest_wait_timeout.argtypes = [vp]
     L.sim_n_params.argtypes = [vp]
     L.sim_n_params.restype = i64
     L.sim_last_error.argtypes = [vp]
@@ -201,6 +202,10 @@ class Simulation:
         cnt = torch.empty((g.numel(),), dtype=torch.int32, device=self.device)
         _check(lib.sim_error_curve(self._h, _ptr(g), g.numel(), _ptr(mean), _ptr(cnt)), self._h)
         return mean.cpu().numpy(), cnt.cpu().numpy()
+
+    def selftest_wait_timeout(self):
+        """Diagnostic: makes a bounded device-side wait run out on this handle (it is unusable afterwards)."""
+        _check(lib.sim_selftest_wait_timeout(self._h), self._h)
 
     def close(self):
         if self._h:

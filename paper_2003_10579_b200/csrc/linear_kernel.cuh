@@ -86,13 +86,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after a few seconds' worth of polls and reports it.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < (1u << 24); ++i) {
+// Bounded wait: gives up after `limit` polls (the default is a few seconds' worth) and reports it.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t limit = 1u << 24) {
+  for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if (i > 4096) __nanosleep(128);
   }
   return false;
+}
+// After a wait has run out: before the block gives up its shared memory, give the row copies that are still in flight
+// a bounded time to land.  At tile (st, parity) the producer is at most one ring ahead: stages st.. complete phase
+// `parity`, stages below st the next one.  A stage that was never issued simply uses up its (short) limit.
+__device__ __forceinline__ void drain_ring(uint64_t* full, int S, int st, uint32_t parity) {
+  for (int s = 0; s < S; ++s) mbar_wait((uint32_t)__cvta_generic_to_shared(&full[s]), s >= st ? parity : parity ^ 1u, 1u << 14);
 }
 // global -> shared bulk copy of `bytes` (multiple of 16, both addresses 16-byte aligned)
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
@@ -262,11 +268,14 @@ __global__ void __launch_bounds__(NT) linear1_kernel(NumericArgs a) {
   int st = 0;             // stage and phase parity of tile `it`, kept as counters (it % S and it / S are 64-bit divisions)
   uint32_t parity = 0;
   for (long long it = 0;; ++it, parity ^= (uint32_t)(st + 1 == S), st = (st + 1 == S ? 0 : st + 1)) {
-    if (!mbar_wait(smem_addr(&full[st]), parity)) { failed = true; break; }
+    // A wait that runs out does not leave on its own: the thread goes on to the tile's block barrier (on whatever the
+    // stage holds - shared memory only, no access depends on it) and the whole block votes there, so that either
+    // every thread of the block drains or none does.
+    const bool ok = mbar_wait(smem_addr(&full[st]), parity);
     const TileInfo ti = info_s[st];
     const float* tile = rows_s + (size_t)st * T * d;
 
-    if (ASYNC && (ti.flags & TILE_FIRST_OF_TASK)) {
+    if (ASYNC && ok && (ti.flags & TILE_FIRST_OF_TASK)) {
       if (ti.snap == cur_slot) {
 #pragma unroll
         for (int e = 0; e < E; ++e) w_tau[e] = w_cur[e];
@@ -316,7 +325,7 @@ __global__ void __launch_bounds__(NT) linear1_kernel(NumericArgs a) {
 #pragma unroll
       for (int q = 0; q < T; ++q) red_s[((it & 1) * NW + warp) * T + q] = part[q];
     }
-    __syncthreads();
+    if (__syncthreads_or(!ok)) { failed = true; break; }
     // every thread is past its reads of the previous tile's stage: refill it
     if (warp == 0) issue_tile(it + S - 1);
 
@@ -424,7 +433,11 @@ __global__ void __launch_bounds__(NT) linear1_kernel(NumericArgs a) {
   }
 
   if (failed) {
-    if (tid == 0) atomicExch(a.err, ERR_WAIT_TIMEOUT);
+    if (tid == 0) {
+      atomicExch(a.err, ERR_WAIT_TIMEOUT);
+      drain_ring(full, S, st, parity);
+    }
+    __syncthreads();
     return;
   }
   if (!ASYNC) {

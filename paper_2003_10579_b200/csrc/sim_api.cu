@@ -319,6 +319,17 @@ sim_status eval_into(sim_handle* h, float* loss) {
   return SIM_OK;
 }
 
+// Self-test of the timeout path: a wait on a barrier that nobody arrives at, with a limit of `limit` polls.  It runs out,
+// the block votes on it and reports through the handle's error word - the steps a numeric kernel takes when one of
+// its bounded waits gives up.  The kernel returns by itself; nothing is left waiting.
+__global__ void wait_timeout_selftest_kernel(int* err, uint32_t limit) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) { mbar_init(smem_addr(&bar), 1); mbar_fence_init(); }
+  __syncthreads();
+  const bool ok = mbar_wait(smem_addr(&bar), 0u, limit);
+  if (__syncthreads_or(!ok) && threadIdx.x == 0) atomicExch(err, ERR_WAIT_TIMEOUT);
+}
+
 __global__ void fill_int_kernel(int* p, int v, int n) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) p[i] = v;
@@ -632,6 +643,13 @@ sim_status sim_error_curve(const sim_handle* h, const double* grid, int32_t n_gr
   error_curve_kernel<<<n_grid, 256, 0, h->stream>>>(h->tr.t, h->tr.loss, h->cap, h->n_updates, h->R, grid, mean_loss, count);
   CUDA_TRY(h, cudaGetLastError());
   CUDA_TRY(h, cudaStreamSynchronize(h->stream));
+  return SIM_OK;
+}
+
+sim_status sim_selftest_wait_timeout(sim_handle* h) {
+  if (!h) return fail(nullptr, SIM_ERR_ARG, "handle is NULL");
+  wait_timeout_selftest_kernel<<<1, 64, 0, h->stream>>>(h->err, 1u << 10);
+  CUDA_TRY(h, cudaGetLastError());
   return SIM_OK;
 }
 

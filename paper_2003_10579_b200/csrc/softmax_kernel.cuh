@@ -156,7 +156,8 @@ __global__ void __launch_bounds__(SMX_NT) softmax_kernel(NumericArgs a) {
   int st = 0;             // stage and phase parity of tile `it`, kept as counters (it % S and it / S are 64-bit divisions)
   uint32_t parity = 0;
   for (long long it = 0;; ++it, parity ^= (uint32_t)(st + 1 == S), st = (st + 1 == S ? 0 : st + 1)) {
-    if (!mbar_wait(smem_addr(&full[st]), parity)) { failed = true; break; }
+    // a wait that runs out is voted on by the whole block, so that every thread drains or none does
+    if (__syncthreads_or(!mbar_wait(smem_addr(&full[st]), parity))) { failed = true; break; }
     const TileInfo ti = info_s[st];
     const float* tile = rows_s + (size_t)st * T * d;
 
@@ -324,7 +325,11 @@ __global__ void __launch_bounds__(SMX_NT) softmax_kernel(NumericArgs a) {
   }
 
   if (failed) {
-    if (tid == 0) atomicExch(a.err, ERR_WAIT_TIMEOUT);
+    if (tid == 0) {
+      atomicExch(a.err, ERR_WAIT_TIMEOUT);
+      drain_ring(full, S, st, parity);
+    }
+    __syncthreads();
     return;
   }
   if (!ASYNC) {

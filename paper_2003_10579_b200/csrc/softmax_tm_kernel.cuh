@@ -32,12 +32,6 @@
 #ifndef SMX_TM_TG
 #define SMX_TM_TG 3
 #endif
-#ifndef SMX_TM_DB
-#define SMX_TM_DB 0
-#endif
-#ifndef SMX_TM_L2
-#define SMX_TM_L2 0
-#endif
 
 namespace ssim {
 
@@ -275,61 +269,22 @@ __global__ void __launch_bounds__(128 * NG) softmax_tm_kernel(NumericArgs a) {
       float acc[NV + 2];
 #pragma unroll
       for (int i = 0; i < NV + 2; ++i) acc[i] = 0.f;
-#if SMX_TM_L2
-      uint64_t acc2[NV];      // (sum over the even features, sum over the odd features) of a logit
-#pragma unroll
-      for (int i = 0; i < NV; ++i) acc2[i] = 0ull;
-#endif
       const float2* rowp = reinterpret_cast<const float2*>(tile + grp * DS) + L;
-#if SMX_TM_DB
-      float wbuf[2][WC];
-      tm_ld20(t_lane, wbuf[0]);
-#endif
 #pragma unroll
       for (int ck = 0; ck < NG * KP; ++ck) {
         const int gp = ck / KP, k = ck % KP;
-#if SMX_TM_DB
-        float* w = wbuf[ck & 1];
-        tm_wait_ld();
-        if (ck + 1 < NG * KP) tm_ld20(t_lane + (ck + 1) * WC, wbuf[(ck + 1) & 1]);
-#else
         float w[WC];
         tm_ld20(t_lane + ck * WC, w);
-#endif
-#if SMX_TM_L2
-        uint64_t x[TG];
-#pragma unroll
-        for (int s = 0; s < TG; ++s) x[s] = reinterpret_cast<const uint64_t*>(rowp)[s * NG * (DS / 2) + 128 * gp + NT * k];
-#else
         float2 x[TG];
 #pragma unroll
         for (int s = 0; s < TG; ++s) x[s] = rowp[s * NG * (DS / 2) + 128 * gp + NT * k];
-#endif
-#if !SMX_TM_DB
         tm_wait_ld();
-#endif
-#if SMX_TM_L2
-#pragma unroll
-        for (int c = 0; c < CP; ++c) {
-          const uint64_t w2 = pack2(w[2 * c], w[2 * c + 1]);
-#pragma unroll
-          for (int s = 0; s < TG; ++s) acc2[s * CP + c] = ffma2(x[s], w2, acc2[s * CP + c]);
-        }
-      }
-#pragma unroll
-      for (int i = 0; i < NV; ++i) {
-        float lo, hi;
-        unpack2(acc2[i], lo, hi);
-        acc[i] = lo + hi;
-      }
-#else
 #pragma unroll
         for (int s = 0; s < TG; ++s)
 #pragma unroll
           for (int c = 0; c < CP; ++c)
             acc[s * CP + c] = fmaf(x[s].y, w[2 * c + 1], fmaf(x[s].x, w[2 * c], acc[s * CP + c]));
       }
-#endif
       tm_reduce_steps<16, NV>(acc, lane);
       if (red_idx >= 0) red_s[warp * 32 + red_idx] = acc[0];
     }
@@ -472,7 +427,10 @@ __global__ void __launch_bounds__(128 * NG) softmax_tm_kernel(NumericArgs a) {
   }
 
   if (failed) {
-    if (tid == 0) atomicExch(a.err, ERR_WAIT_TIMEOUT);
+    if (tid == 0) {
+      atomicExch(a.err, ERR_WAIT_TIMEOUT);
+      drain_ring(full, S, st, parity);
+    }
   } else if (!ASYNC && my_iters > 0) {
     float* dst = a.w_state + (size_t)r * np;
 #pragma unroll

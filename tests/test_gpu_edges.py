@@ -79,3 +79,45 @@ def test_more_workers_than_warp_lanes(B, variant):
     run_case(B, inputs.make_logistic(500, 12, 0.05, 62), variant=variant, P=128, K=17, m=3, eta=0.05, R=2, J=30, use_ref=False)
     run_case(B, inputs.make_mixture(400, 20, 4, 0.5, 63, "softmax"), variant=variant, P=70, K=33, m=2, eta=0.05, R=2, J=20,
              use_ref=False)
+
+
+def test_a_wait_that_runs_out_is_reported_and_poisons_only_its_handle(B):
+    """The timeout path end to end, without hanging anything: the library's self-test kernel waits about a thousand
+    polls on a barrier nobody arrives at and gives up; the handle's next synchronising call must return
+    SIM_ERR_TIMEOUT, the handle must then refuse to run, and another handle on the same device must be unaffected."""
+    data = to_device(inputs.make_lsq(300, 16, 0.1, 56))
+    kw = dict(P=4, K=2, variant="ksync", delay_kind="exp", mu=1.0, eta=0.05, m=4, seed=1, n_replicas=3)
+    bad, good = B.Simulation(data, **kw), B.Simulation(data, **kw)
+    bad.run(5)
+    good.run(5)
+    bad.selftest_wait_timeout()
+    with pytest.raises(B.SimError) as e:
+        bad.trace_size()
+    assert e.value.status == 4 and "wait ran out" in str(e.value)          # SIM_ERR_TIMEOUT
+    with pytest.raises(B.SimError) as e:
+        bad.run(1)
+    assert e.value.status == 5                                             # SIM_ERR_STATE: the handle is poisoned
+    with pytest.raises(B.SimError) as e:
+        bad.params()
+    assert e.value.status == 4
+    bad.close()
+    good.run(5)                                                            # the device and other handles carry on
+    tr = good.trace()
+    assert tr["t"].shape == (3, 10) and np.isfinite(tr["loss"]).all()
+    good.close()
+
+
+def test_switching_the_k_schedule_off_also_leaves_the_loss_driven_mode(B):
+    """sim_set_adasync_loss followed by sim_set_adasync(0, 0): fixed K again, trace rows K wide, the fixed-K schedule."""
+    data = to_device(inputs.make_lsq(300, 16, 0.1, 57))
+    kw = dict(P=6, K=2, variant="kasync", delay_kind="exp", mu=1.0, eta=0.05, m=4, seed=2, n_replicas=4)
+    a, b = B.Simulation(data, **kw), B.Simulation(data, **kw)
+    a.set_adasync_loss(1, 3.0)
+    a.set_adasync(0, 0.0)
+    a.run(30)
+    b.run(30)
+    assert a.trace_size() == (30, 2)
+    ta, tb = a.trace(), b.trace()
+    for k in ta:
+        assert np.array_equal(ta[k], tb[k]), k
+    a.close(); b.close()
