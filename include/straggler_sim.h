@@ -115,7 +115,8 @@ sim_status sim_set_adasync(sim_handle* h, int32_t K0, double t_interval);
  *   K-sync:  the positive root of  K^2 / (P - K) = K0^2 / (P - K0) * F(w_0) / F(w_start)
  * rounded half up, never decreasing, at most P.  Replicas pause at different updates, so sim_run
  * proceeds in rounds (one per interval crossing) and synchronises the stream between rounds.  LSQ,
- * LOGISTIC and SOFTMAX only (the rule needs sim_eval_loss).  Only before the first sim_run.
+ * LOGISTIC and SOFTMAX only (the MLP's kernels advance all replicas in lock step and cannot pause them one by
+ * one).  Only before the first sim_run.
  */
 sim_status sim_set_adasync_loss(sim_handle* h, int32_t K0, double t_interval);
 
@@ -158,11 +159,46 @@ sim_status sim_get_params(const sim_handle* h, float* w);
 /*
  * Full-data empirical risk F(w_j) = (1/N) sum_n f(w_j, xi_n) (Eq. 1) of every replica's current
  * parameters into a DEVICE buffer [R]: the "error" of Section 2.3, for error-versus-wall-clock
- * curves (call it between sim_run calls; the clock of the same update is in the trace).  One dense
- * product over all replicas, fp32 logits, fp64 sums in a fixed order.  Built for LSQ, LOGISTIC and
- * SOFTMAX (SIM_ERR_ARG otherwise).  Enqueued on the handle's stream; does not wait.
+ * curves (call it between sim_run calls; the clock of the same update is in the trace).  Linear
+ * models: one dense product over all replicas, fp32 logits, fp64 sums in a fixed order.  MLP2: the
+ * tensor-core forward pass (bf16 operands x and W1, as in the gradients) over all rows, fp64 sums in a
+ * fixed order.  SIM_ERR_ARG for SIM_NONE.  Enqueued on the handle's stream; does not wait.
  */
 sim_status sim_eval_loss(sim_handle* h, float* loss);
+
+/*
+ * Error against wall clock, the two metrics of Section 2.3 recorded together inside sim_run: with every > 0 the
+ * full-data risk F(w_j) (Eq. 1, as sim_eval_loss computes it) of every replica is recorded before the first update
+ * (entry 0: F(w_0) at time 0) and after every `every`-th update (entry i: after i * every updates, at the clock of
+ * that update), whatever the lengths of the sim_run calls.  every = 0 switches it off.  Only before the first
+ * sim_run; not together with sim_set_adasync_loss (SIM_ERR_STATE); SIM_ERR_ARG for SIM_NONE.  One evaluation reads
+ * the whole data set: choose `every` accordingly.
+ */
+sim_status sim_set_eval_every(sim_handle* h, int64_t every);
+
+/* Number of recorded evaluations E (0 before the first sim_run with a risk trace). */
+sim_status sim_risk_trace_size(const sim_handle* h, int64_t* n_evals);
+
+/* The risk trace and its clock into caller-owned DEVICE buffers [R][E] (either may be NULL); synchronises the stream. */
+sim_status sim_get_risk_trace(const sim_handle* h, float* risk /*[R][E]*/, double* t /*[R][E]*/);
+
+/*
+ * The error-runtime curve of Section 2.3 from the risk trace: for each grid time g (DEVICE [n_grid]) the mean over
+ * replicas of F(w) - f_star at the replica's last evaluation completed by g (f_star: the caller's F*, e.g. from the
+ * normal equations for LSQ; 0 to get the risk itself) and the number of replicas counted (all of them from g = 0 on,
+ * since entry 0 is at time 0).  DEVICE outputs [n_grid]; synchronises.  SIM_ERR_STATE without a risk trace.
+ */
+sim_status sim_risk_curve(const sim_handle* h, const double* grid, int32_t n_grid, float f_star, float* mean_err, int32_t* count);
+
+/*
+ * The trade-off across K that motivates AdaSync (Sections 1, 5 and 6: a small K is ahead early, a large K reaches a
+ * lower floor): the lower envelope of the risk curves of several simulations of the same problem (typically one
+ * handle per K) on a common grid.  env[g] = the smallest mean error at grid time g among the handles, best[g] = the
+ * index of the handle that attains it (lowest index on ties).  grid, env, best are DEVICE arrays [n_grid]; every
+ * handle needs a risk trace.  Allocates and frees two temporary arrays; synchronises every handle's stream.
+ */
+sim_status sim_risk_envelope(sim_handle* const* handles, int32_t n_handles, const double* grid, int32_t n_grid, float f_star,
+                             float* env, int32_t* best);
 
 /*
  * Error against simulated wall clock on a common time grid - the error-runtime trade-off picture of

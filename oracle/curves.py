@@ -19,3 +19,17 @@ def error_curve(t, err, grid):
                 count[i] += 1
         mean[i] = total / count[i] if count[i] else 0.0
     return mean, count
+
+
+def envelope(curves, counts):
+    """Lower envelope of several error curves on one grid: curves, counts [n, G].  At each grid point the smallest
+    value among the curves that have data there (count > 0) and the index of that curve (the lowest index on
+    ties); where no curve has data the value is 0 and the index -1."""
+    curves, counts = np.asarray(curves, np.float64), np.asarray(counts)
+    n, G = curves.shape
+    env, best = np.zeros(G), np.full(G, -1, np.int32)
+    for g in range(G):
+        for c in range(n):
+            if counts[c, g] > 0 and (best[g] < 0 or curves[c, g] < env[g]):
+                env[g], best[g] = curves[c, g], c
+    return env, best

@@ -20,7 +20,8 @@ STATUS = {0: "SIM_OK", 1: "SIM_ERR_ARG", 2: "SIM_ERR_ALLOC", 3: "SIM_ERR_CUDA", 
           5: "SIM_ERR_STATE", 6: "SIM_ERR_INTERNAL"}
 
 EXPORTS = ["sim_create", "sim_set_params", "sim_set_adasync", "sim_set_adasync_loss", "sim_set_tuning", "sim_reserve", "sim_run",
-           "sim_trace_size", "sim_get_trace", "sim_get_params", "sim_eval_loss", "sim_error_curve", "sim_selftest_wait_timeout", "sim_n_params", "sim_last_error",
+           "sim_trace_size", "sim_get_trace", "sim_get_params", "sim_eval_loss", "sim_error_curve", "sim_set_eval_every", "sim_risk_trace_size",
+           "sim_get_risk_trace", "sim_risk_curve", "sim_risk_envelope", "sim_selftest_wait_timeout", "sim_n_params", "sim_last_error",
            "sim_destroy", "sim_draw_delays", "sim_draw_indices", "sim_simulate_host", "sim_sweep_host", "sim_schedule_noalloc",
            "sim_noalloc_last_error"]
 
@@ -61,6 +62,11 @@ def _load():
     L.sim_eval_loss.argtypes = [vp, vp]
     L.sim_error_curve.argtypes = [vp, vp, i32, vp, vp]
     L.sim_selftest_wait_timeout.argtypes = [vp]
+    L.sim_set_eval_every.argtypes = [vp, i64]
+    L.sim_risk_trace_size.argtypes = [vp, C.POINTER(i64)]
+    L.sim_get_risk_trace.argtypes = [vp, vp, vp]
+    L.sim_risk_curve.argtypes = [vp, vp, i32, C.c_float, vp, vp]
+    L.sim_risk_envelope.argtypes = [C.POINTER(vp), i32, vp, i32, C.c_float, vp, vp]
     L.sim_n_params.argtypes = [vp]
     L.sim_n_params.restype = i64
     L.sim_last_error.argtypes = [vp]
@@ -203,6 +209,27 @@ class Simulation:
         _check(lib.sim_error_curve(self._h, _ptr(g), g.numel(), _ptr(mean), _ptr(cnt)), self._h)
         return mean.cpu().numpy(), cnt.cpu().numpy()
 
+    def set_eval_every(self, every):
+        """Record the full-data risk of every replica before the first and after every `every`-th update."""
+        _check(lib.sim_set_eval_every(self._h, every), self._h)
+
+    def risk_trace(self, to_numpy=True):
+        """(risk [R, E], t [R, E]): entry 0 is F(w_0) at time 0, entry i the risk after i * every updates."""
+        E = C.c_int64()
+        _check(lib.sim_risk_trace_size(self._h, C.byref(E)), self._h)
+        risk = torch.empty((self.R, E.value), dtype=torch.float32, device=self.device)
+        t = torch.empty((self.R, E.value), dtype=torch.float64, device=self.device)
+        _check(lib.sim_get_risk_trace(self._h, _ptr(risk), _ptr(t)), self._h)
+        return (risk.cpu().numpy(), t.cpu().numpy()) if to_numpy else (risk, t)
+
+    def risk_curve(self, grid, f_star=0.0):
+        """Mean over replicas of F(w) - f_star against simulated wall clock at the times in `grid`."""
+        g = torch.as_tensor(np.asarray(grid, np.float64)).to(self.device)
+        mean = torch.empty((g.numel(),), dtype=torch.float32, device=self.device)
+        cnt = torch.empty((g.numel(),), dtype=torch.int32, device=self.device)
+        _check(lib.sim_risk_curve(self._h, _ptr(g), g.numel(), f_star, _ptr(mean), _ptr(cnt)), self._h)
+        return mean.cpu().numpy(), cnt.cpu().numpy()
+
     def selftest_wait_timeout(self):
         """Diagnostic: makes a bounded device-side wait run out on this handle (it is unusable afterwards)."""
         _check(lib.sim_selftest_wait_timeout(self._h), self._h)
@@ -217,6 +244,18 @@ class Simulation:
             self.close()
         except Exception:
             pass
+
+
+def risk_envelope(sims, grid, f_star=0.0):
+    """Lower envelope over several simulations' risk curves on a common grid: (env [G], best [G])."""
+    dev = sims[0].device
+    g = torch.as_tensor(np.asarray(grid, np.float64)).to(dev)
+    env = torch.empty((g.numel(),), dtype=torch.float32, device=dev)
+    best = torch.empty((g.numel(),), dtype=torch.int32, device=dev)
+    hs = (C.c_void_p * len(sims))(*[s._h for s in sims])
+    st = lib.sim_risk_envelope(hs, len(sims), _ptr(g), g.numel(), f_star, _ptr(env), _ptr(best))
+    _check(st)
+    return env.cpu().numpy(), best.cpu().numpy()
 
 
 def draw_delays(delay_kind, mu, shift, seed, replica_base, n_replicas, P, n_seq):

@@ -51,6 +51,12 @@ struct MlpArgs {
   MlpScratch sc;
   int H, P;
   long long j;            // update being processed
+  // forward-only evaluation of the full-data risk (the forward kernel's EVAL form): consecutive 128-row blocks of the
+  // data set instead of minibatches, every replica at its current version
+  int eval_blocks;              // ceil(n / 128)
+  const uint8_t* eval_slot;     // [R] pool slot of the current version (asynchronous variants) or null:
+  int eval_parity;              //     then every replica's current version sits in slot eval_parity
+  float* eval_part;             // [R][eval_blocks][4] loss sums per 32-row group
 };
 
 inline const char* mlp_shape_unsupported(int d, int H, int C, int m) {

@@ -105,22 +105,31 @@ inline __host__ __device__ TcLayout tc_forward_layout(int H) {
   return L;
 }
 
+// EVAL = true is the forward-only form for the full-data risk F(w) of Eq. 1: one CTA per (replica, 128 consecutive rows
+// of the data set), the replica's current version, and only the rows' losses leave the CTA.
+template <bool EVAL>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmW, MlpArgs g) {
   const NumericArgs& a = g.na;
   const MlpScratch& sc = g.sc;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int H = sc.H, C = sc.C, d = sc.d, m = sc.m;
-  const int mtiles = m / 128;
+  const int mtiles = EVAL ? g.eval_blocks : m / 128;
   const int mt = blockIdx.x % mtiles;
-  const int l = (blockIdx.x / mtiles) % sc.Kmax;
-  const int r = blockIdx.x / (mtiles * sc.Kmax);
+  const int l = EVAL ? 0 : (blockIdx.x / mtiles) % sc.Kmax;
+  const int r = EVAL ? blockIdx.x / mtiles : blockIdx.x / (mtiles * sc.Kmax);
   const long long j = g.j;
-  const int K = (int)a.K_used[(size_t)r * a.cap + j];
-  if (l >= K) return;
-  const size_t ent = ((size_t)r * a.cap + j) * a.K_stride + l;
-  const uint32_t worker = a.worker[ent], seq = a.seq[ent];
-  const int snap = mlp_snap_slot(a, r, j, l);
+  uint32_t worker = 0, seq = 0;
+  int snap;
+  if (EVAL) {
+    snap = g.eval_slot ? (int)g.eval_slot[r] : g.eval_parity;
+  } else {
+    const int K = (int)a.K_used[(size_t)r * a.cap + j];
+    if (l >= K) return;
+    const size_t ent = ((size_t)r * a.cap + j) * a.K_stride + l;
+    worker = a.worker[ent]; seq = a.seq[ent];
+    snap = mlp_snap_slot(a, r, j, l);
+  }
   const uint32_t rid = a.replica_base + (uint32_t)r;
   const size_t task = (size_t)r * sc.Kmax + l;
   const long long dH = (long long)d * H;
@@ -169,8 +178,14 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmW, MlpArgs g) {
   if (warp == 1) tc_alloc(smem_addr(tmem_slot), tmem_cols);
   if (tid >= 64 && tid < 192) {                     // the minibatch: sample rows and labels (the A producers need them first)
     const int t = tid - 64;
-    uint32_t idx = draw_index(a.seed, rid, worker, seq, (uint32_t)(mt * 128 + t), a.n);
-    if ((uint64_t)idx >= a.n) { atomicExch(a.err, ERR_BAD_INDEX); idx = 0; }
+    uint32_t idx;
+    if (EVAL) {     // consecutive rows; a row past the end of the data set repeats the last one and is left out of the sum
+      const uint64_t want = (uint64_t)mt * 128 + t;
+      idx = (uint32_t)(want < a.n ? want : a.n - 1);
+    } else {
+      idx = draw_index(a.seed, rid, worker, seq, (uint32_t)(mt * 128 + t), a.n);
+      if ((uint64_t)idx >= a.n) { atomicExch(a.err, ERR_BAD_INDEX); idx = 0; }
+    }
     rows_s[t] = (int)idx;
     label_s[t] = reinterpret_cast<const int*>(a.y)[idx];
   }
@@ -296,7 +311,7 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmW, MlpArgs g) {
               }
             }
           }
-          hout[i4] = make_float4(hv[0], hv[1], hv[2], hv[3]);
+          if (!EVAL) hout[i4] = make_float4(hv[0], hv[1], hv[2], hv[3]);
         }
       }
 #pragma unroll
@@ -323,6 +338,13 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmW, MlpArgs g) {
       float sexcl = 0.f;
 #pragma unroll
       for (int c = 0; c < 16; ++c) { z[c] = (c < C && c != cmax) ? expf(z[c] - zmax) : 0.f; sexcl += z[c]; }
+      if (EVAL) {     // the row's loss is all that is wanted
+        if (!ehalf) {
+          const bool real = (uint64_t)mt * 128 + row < a.n;
+          const float rowloss = warp_sum(real ? log1pf(sexcl) + (zmax - zl) : 0.f);
+          if (lane == 0) g.eval_part[((size_t)r * g.eval_blocks + mt) * 4 + q] = rowloss;
+        }
+      } else {
       const float ssum = 1.f + sexcl;
       float d2[16];
 #pragma unroll
@@ -375,6 +397,7 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmW, MlpArgs g) {
         }
         warp_transpose_reduce(dv, lane);
         sc.db1_part[(task * parts + part) * H + ch * 32 + lane] = dv[0];
+      }
       }
     }
   }
@@ -737,20 +760,53 @@ inline bool tc_make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64
 
 struct MlpMaps { CUtensorMap tmW, tmD; bool ready = false; };
 
+inline bool mlp_make_maps(MlpScratch& s, MlpMaps& maps) {
+  if (maps.ready) return true;
+  const int n_halves = s.H > 256 ? 2 : 1;
+  if (!tc_make_map(&maps.tmW, s.W1qT, (uint64_t)s.R * s.n_slots * (s.d / TC_BK) * s.H, (uint64_t)TC_BK, TC_BK, (uint32_t)(s.H / n_halves)) ||
+      !tc_make_map(&maps.tmD, s.D1q, (uint64_t)s.R * s.Kmax * s.m, (uint64_t)s.H, 64, 64))
+    return false;
+  maps.ready = true;
+  return true;
+}
+
+// sum of a replica's per-group loss sums, in fp64 and a fixed order (lane-strided, then a shuffle tree), over n samples
+__global__ void mlp_eval_finish_kernel(const float* part, int R, int per_replica, long long n, float* out) {
+  const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (r >= R) return;
+  double s = 0.0;
+  for (int i = lane; i < per_replica; i += 32) s += (double)part[(size_t)r * per_replica + i];
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
+  if (lane == 0) out[r] = (float)(s / (double)n);
+}
+
+// Full-data risk of every replica's current version: the forward kernel over all rows of the data set, losses only.
+inline cudaError_t run_mlp_eval(NumericArgs& a, MlpScratch& s, MlpMaps& maps, const uint8_t* cur_slot, int parity, float* part,
+                                float* out, cudaStream_t stream, const char** why) {
+  *why = nullptr;
+  if (!mlp_make_maps(s, maps)) { *why = "mlp: could not encode the TMA tensor maps"; return cudaSuccess; }
+  cudaError_t e;
+  const TcLayout L = tc_forward_layout(s.H);
+  if ((e = cudaFuncSetAttribute(mlp_forward_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total)) != cudaSuccess) return e;
+  MlpArgs g{};
+  g.na = a; g.sc = s; g.H = s.H; g.P = 0; g.j = 0;
+  g.eval_blocks = (int)((s.n + 127) / 128); g.eval_slot = cur_slot; g.eval_parity = parity; g.eval_part = part;
+  mlp_forward_tc_kernel<true><<<a.R * g.eval_blocks, TC_THREADS, L.total, stream>>>(maps.tmW, g);
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  mlp_eval_finish_kernel<<<(a.R + 3) / 4, 128, 0, stream>>>(part, a.R, g.eval_blocks * 4, s.n, out);
+  return cudaGetLastError();
+}
+
 inline cudaError_t run_mlp(NumericArgs& a, MlpScratch& s, MlpMaps& maps, int P, cudaStream_t stream, const char** why) {
   *why = nullptr;
   cudaError_t e;
-  const int n_halves = s.H > 256 ? 2 : 1;
-  if (!maps.ready) {
-    if (!tc_make_map(&maps.tmW, s.W1qT, (uint64_t)s.R * s.n_slots * (s.d / TC_BK) * s.H, (uint64_t)TC_BK, TC_BK, (uint32_t)(s.H / n_halves)) ||
-        !tc_make_map(&maps.tmD, s.D1q, (uint64_t)s.R * s.Kmax * s.m, (uint64_t)s.H, 64, 64)) {
-      *why = "mlp: could not encode the TMA tensor maps";
-      return cudaSuccess;
-    }
-    maps.ready = true;
+  if (!mlp_make_maps(s, maps)) {
+    *why = "mlp: could not encode the TMA tensor maps";
+    return cudaSuccess;
   }
   const TcLayout L = tc_forward_layout(s.H);
-  if ((e = cudaFuncSetAttribute(mlp_forward_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(mlp_forward_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total)) != cudaSuccess) return e;
   const TcDw1Layout LD = tc_dw1_layout(s.H);
   if ((e = cudaFuncSetAttribute(mlp_dw1_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, LD.total)) != cudaSuccess) return e;
   int dev = 0, sms = 148;
@@ -764,7 +820,7 @@ inline cudaError_t run_mlp(NumericArgs& a, MlpScratch& s, MlpMaps& maps, int P, 
   for (long long u = 0; u < a.iters; ++u) {
     g.j = a.j0 + u;
     mlp_rows_kernel<<<a.R * s.Kmax, 128, 0, stream>>>(g);
-    mlp_forward_tc_kernel<<<a.R * s.Kmax * mtiles, TC_THREADS, L.total, stream>>>(maps.tmW, g);
+    mlp_forward_tc_kernel<false><<<a.R * s.Kmax * mtiles, TC_THREADS, L.total, stream>>>(maps.tmW, g);
     mlp_head_kernel<<<a.R * (s.H / 32), MLP_HEAD_THREADS, 0, stream>>>(g);
     mlp_dw1_tc_kernel<<<dw1_grid, DW1_THREADS, LD.total, stream>>>(maps.tmD, g);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;

@@ -73,6 +73,10 @@ struct sim_handle {
   float* F0 = nullptr; float* Fcur = nullptr;
   long long* done = nullptr; long long* run_j0 = nullptr; long long* run_iters = nullptr; long long* q_last = nullptr;
   int* K_cur = nullptr; int* want_eval = nullptr; int* remaining = nullptr;
+  // full-data risk recorded inside sim_run: entry 0 is F(w_0), entry i the risk after i * eval_every updates
+  long long eval_every = 0, n_evals = 0, risk_cap = 0;
+  float* risk = nullptr;            // [risk_cap][R]
+  float* mlp_eval_part = nullptr;   // MLP: per 32-row group partial loss sums of one evaluation
   TraceBuffers tr;
   bool poisoned = false;
   bool in_arena = false;      // buffers come from the creating thread's DeviceArena and are not freed one by one
@@ -293,13 +297,38 @@ void free_all(sim_handle* h) {
   cudaFree(h->run_iters); cudaFree(h->q_last); cudaFree(h->K_cur); cudaFree(h->want_eval); cudaFree(h->remaining);
   cudaFree(h->tr.t); cudaFree(h->tr.loss); cudaFree(h->tr.dist2); cudaFree(h->tr.K_used);
   cudaFree(h->tr.worker); cudaFree(h->tr.stale); cudaFree(h->tr.seq); cudaFree(h->tr.snap_slot);
-  cudaFree(h->tr.new_slot);
+  cudaFree(h->tr.new_slot); cudaFree(h->risk); cudaFree(h->mlp_eval_part);
+}
+
+// MLP: bf16 copy of the data, per-update scratch and the bf16 shadow of the initial W1, made on first use
+cudaError_t ensure_mlp_scratch(sim_handle* h) {
+  if (h->mlp.Xq) return cudaSuccess;
+  cudaError_t ce = mlp_scratch_alloc(h->mlp, h->prob.X, h->prob.n, h->prob.d, h->prob.hidden, h->prob.n_classes, h->m,
+                                     h->K_stride, h->R, h->n_slots, h->stream);
+  if (ce == cudaSuccess) ce = mlp_after_set_params(h->mlp, h->pool, h->slot_stride, h->stream);
+  return ce;
 }
 
 sim_status eval_into(sim_handle* h, float* loss) {
   const sim_model mdl = h->prob.model;
+  if (mdl == SIM_MLP2) {
+    // forward pass of the tensor-core kernel over the whole data set, every replica at its current version
+    const int blocks = (int)((h->prob.n + 127) / 128);
+    if (!h->mlp_eval_part) CUDA_TRY(h, dev_alloc(&h->mlp_eval_part, (size_t)h->R * blocks * 4, h->stream, false));
+    CUDA_TRY(h, ensure_mlp_scratch(h));
+    NumericArgs a{};
+    a.X = h->prob.X; a.y = h->prob.label; a.n = (uint64_t)h->prob.n; a.d = h->prob.d; a.m = h->m; a.model = (int)mdl;
+    a.n_classes = h->prob.n_classes; a.replica_base = h->replica_base; a.R = h->R; a.is_async = h->is_async ? 1 : 0;
+    a.n_slots = h->n_slots; a.n_params = h->n_params; a.slot_stride = h->slot_stride; a.pool = h->pool; a.err = h->err;
+    const char* why = nullptr;
+    const cudaError_t ce = run_mlp_eval(a, h->mlp, h->mlp_maps, h->is_async ? h->cur_slot : nullptr, (int)(h->n_updates & 1),
+                                        h->mlp_eval_part, loss, h->stream, &why);
+    if (why) return fail(h, SIM_ERR_ARG, why);
+    CUDA_TRY(h, ce);
+    return SIM_OK;
+  }
   if (mdl != SIM_LSQ && mdl != SIM_LOGISTIC && mdl != SIM_SOFTMAX)
-    return fail(h, SIM_ERR_ARG, "the full-data risk is built for the linear models (LSQ, logistic, softmax)");
+    return fail(h, SIM_ERR_ARG, "the full-data risk needs a model (LSQ, logistic, softmax or the MLP)");
   EvalArgs e{};
   e.X = h->prob.X;
   e.y = mdl == SIM_LSQ ? static_cast<const void*>(h->prob.y) : static_cast<const void*>(h->prob.label);
@@ -330,12 +359,140 @@ __global__ void wait_timeout_selftest_kernel(int* err, uint32_t limit) {
   if (__syncthreads_or(!ok) && threadIdx.x == 0) atomicExch(err, ERR_WAIT_TIMEOUT);
 }
 
+// risk trace [evals][R] (as recorded) -> [R][evals] for the caller, with the clock of each evaluation: entry 0 is
+// F(w_0) at time 0, entry i the risk after i * every updates, i.e. at the time recorded for update i * every - 1
+__global__ void risk_trace_out_kernel(const float* risk, const double* t, long long cap, long long every, int R, long long E,
+                                      float* risk_out, double* t_out) {
+  const long long total = (long long)R * E;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const long long r = i / E, e = i % E;
+    if (risk_out) risk_out[i] = risk[e * R + r];
+    if (t_out) t_out[i] = e == 0 ? 0.0 : t[r * cap + e * every - 1];
+  }
+}
+
+// Mean over replicas of F(w) - f_star at the replica's last evaluation completed by grid time g (one block per grid
+// point, binary search over the evaluation times, fp64 tree sum in a fixed order).
+__global__ void __launch_bounds__(256) risk_curve_kernel(const float* risk, const double* t, long long cap, long long every, int R,
+                                                         long long E, const double* grid, float f_star, float* mean, int* count) {
+  __shared__ double sum_s[256];
+  __shared__ int cnt_s[256];
+  const double g = grid[blockIdx.x];
+  double s = 0.0;
+  int c = 0;
+  for (int r = threadIdx.x; r < R; r += 256) {
+    const double* tr = t + (size_t)r * cap;
+    long long lo = 0, hi = E;                 // first evaluation with time > g (evaluation 0 is at time 0)
+    while (lo < hi) {
+      const long long mid = (lo + hi) >> 1;
+      const double tm = mid == 0 ? 0.0 : tr[mid * every - 1];
+      if (tm <= g) lo = mid + 1; else hi = mid;
+    }
+    if (lo > 0) { s += (double)risk[(lo - 1) * R + r] - (double)f_star; ++c; }
+  }
+  sum_s[threadIdx.x] = s; cnt_s[threadIdx.x] = c;
+  __syncthreads();
+  for (int off = 128; off > 0; off >>= 1) {
+    if ((int)threadIdx.x < off) { sum_s[threadIdx.x] += sum_s[threadIdx.x + off]; cnt_s[threadIdx.x] += cnt_s[threadIdx.x + off]; }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) { count[blockIdx.x] = cnt_s[0]; mean[blockIdx.x] = cnt_s[0] ? (float)(sum_s[0] / cnt_s[0]) : 0.f; }
+}
+
+// Lower envelope of n curves on one grid: at each grid point the smallest value among the curves that have data
+// there (count > 0), and which curve it belongs to (lowest index on ties; -1 and 0 where no curve has data).
+__global__ void envelope_kernel(const float* curves, const int* counts, int n, int G, float* env, int* best) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= G) return;
+  float v = 0.f;
+  int b = -1;
+  for (int c = 0; c < n; ++c)
+    if (counts[(size_t)c * G + i] > 0 && (b < 0 || curves[(size_t)c * G + i] < v)) { v = curves[(size_t)c * G + i]; b = c; }
+  env[i] = v;
+  best[i] = b;
+}
+
 __global__ void fill_int_kernel(int* p, int v, int n) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) p[i] = v;
 }
 
 }  // namespace
+
+// One stretch of `iters` updates of every replica: the arrival process, then the arithmetic along it (in rounds when
+// the loss-driven K rule pauses replicas at interval boundaries).  Capacity has been checked by the caller.
+static sim_status run_span(sim_handle* h, int64_t iters) {
+  sim_status st = SIM_OK;
+  ScheduleArgs sa{};
+  sa.variant = h->variant; sa.P = h->P; sa.K_fixed = h->K; sa.K0 = h->K0; sa.t_interval = h->t_interval;
+  sa.law.kind = (int)h->delay.kind; sa.law.mu = h->delay.mu; sa.law.shift = h->delay.shift;
+  sa.seed = h->seed; sa.R = h->R; sa.replica_base = h->replica_base;
+  sa.j0 = h->n_updates; sa.iters = iters; sa.cap = h->cap; sa.K_stride = h->K_stride; sa.n_slots = h->n_slots;
+  sa.s = h->s; sa.tau = h->tau; sa.f = h->f; sa.wslot = h->wslot; sa.cur_slot = h->cur_slot;
+  sa.begin_slot = h->begin_slot; sa.clock = h->clock;
+  sa.t = h->tr.t; sa.K_used = h->tr.K_used; sa.worker = h->tr.worker; sa.stale = h->tr.stale; sa.seq = h->tr.seq;
+  sa.snap_slot = h->tr.snap_slot; sa.new_slot = h->tr.new_slot; sa.err = h->err;
+  // Loss-driven K: replicas pause where an update starts in a new interval and K may still grow; each
+  // round schedules every replica up to its next pause (or the target), runs the arithmetic that far,
+  // evaluates the full-data risk and sets the paused replicas' new K.  Rounds = interval crossings + 1.
+  const bool adaptive = h->ada_loss && h->t_interval > 0.0;
+  if (adaptive) {
+    if (!h->F0_ready) { if ((st = eval_into(h, h->F0)) != SIM_OK) return st; h->F0_ready = true; }
+    sa.adaptive = 1; sa.target = h->n_updates + iters; sa.done = h->done; sa.run_j0 = h->run_j0; sa.run_iters = h->run_iters;
+    sa.K_cur = h->K_cur; sa.q_last = h->q_last; sa.want_eval = h->want_eval;
+  }
+  for (long long round = 0;; ++round) {
+  CUDA_TRY(h, launch_schedule(sa, h->stream));
+
+  if (h->prob.model != SIM_NONE) {
+    NumericArgs a{};
+    if (adaptive) { a.run_j0 = h->run_j0; a.run_iters = h->run_iters; }
+    a.X = h->prob.X;
+    a.y = h->prob.model == SIM_LSQ ? static_cast<const void*>(h->prob.y) : static_cast<const void*>(h->prob.label);
+    a.w_ref = h->prob.w_ref; a.n = (uint64_t)h->prob.n; a.d = h->prob.d; a.m = h->m; a.model = (int)h->prob.model;
+    a.n_classes = h->prob.n_classes; a.eta = h->eta; a.seed = h->seed; a.replica_base = h->replica_base; a.R = h->R;
+    a.j0 = h->n_updates; a.iters = iters; a.cap = h->cap; a.K_stride = h->K_stride; a.is_async = h->is_async ? 1 : 0;
+    a.n_slots = h->n_slots; a.n_params = h->n_params; a.slot_stride = h->slot_stride;
+    a.K_used = h->tr.K_used; a.worker = h->tr.worker; a.seq = h->tr.seq; a.snap_slot = h->tr.snap_slot;
+    a.new_slot = h->tr.new_slot; a.begin_slot = h->begin_slot; a.loss = h->tr.loss; a.dist2 = h->tr.dist2;
+    a.w_state = h->w_state; a.pool = h->pool; a.err = h->err;
+    const char* why = nullptr;
+    cudaError_t ce = cudaSuccess;
+    switch (h->prob.model) {
+      case SIM_LSQ: case SIM_LOGISTIC: st = run_linear1(h, a); break;
+      case SIM_SOFTMAX:
+        ce = run_softmax_any(a, h->tune_stages, h->stream, &why);
+        st = why ? fail(h, SIM_ERR_ARG, why) : SIM_OK;
+        break;
+      case SIM_MLP2:
+        ce = ensure_mlp_scratch(h);
+        if (ce == cudaSuccess) ce = run_mlp(a, h->mlp, h->mlp_maps, h->P, h->stream, &why);
+        if (ce == cudaSuccess && !h->is_async)   // synchronous variants ping-pong between two slots
+          ce = cudaMemsetAsync(h->cur_slot, (int)((h->n_updates + iters) & 1), (size_t)h->R, h->stream);
+        st = why ? fail(h, SIM_ERR_ARG, why) : SIM_OK;
+        break;
+      default: st = fail(h, SIM_ERR_ARG, "unknown model");
+    }
+    if (ce != cudaSuccess) st = fail(h, SIM_ERR_CUDA, std::string("numeric kernel launch: ") + cudaGetErrorString(ce));
+    if (st != SIM_OK) { h->poisoned = true; return st; }
+  }
+  if (!adaptive) break;
+  if ((st = eval_into(h, h->Fcur)) != SIM_OK) { h->poisoned = true; return st; }
+  CUDA_TRY(h, cudaMemsetAsync(h->remaining, 0, sizeof(int), h->stream));
+  adasync_update_kernel<<<(h->R + 127) / 128, 128, 0, h->stream>>>(h->variant, h->P, h->K0, h->t_interval, h->R, sa.target, h->F0,
+                                                                  h->Fcur, h->clock, h->done, h->K_cur, h->q_last, h->want_eval,
+                                                                  h->remaining);
+  CUDA_TRY(h, cudaGetLastError());
+  int remaining = 0;
+  CUDA_TRY(h, cudaMemcpyAsync(&remaining, h->remaining, sizeof(int), cudaMemcpyDeviceToHost, h->stream));
+  CUDA_TRY(h, cudaStreamSynchronize(h->stream));
+  if (remaining == 0) break;
+  if (round > iters + 8) { h->poisoned = true; return fail(h, SIM_ERR_INTERNAL, "loss-driven K: no progress"); }
+  }
+  h->n_updates += iters;
+  return SIM_OK;
+}
+
 
 extern "C" {
 
@@ -478,78 +635,33 @@ sim_status sim_run(sim_handle* h, int64_t iters) {
   if (h->n_updates + iters > (1ll << 31)) return fail(h, SIM_ERR_ARG, "more than 2^31 updates");
   sim_status st = ensure_capacity(h, h->n_updates + iters);
   if (st != SIM_OK) return st;
+  if (h->eval_every <= 0) return run_span(h, iters);
 
-  ScheduleArgs sa{};
-  sa.variant = h->variant; sa.P = h->P; sa.K_fixed = h->K; sa.K0 = h->K0; sa.t_interval = h->t_interval;
-  sa.law.kind = (int)h->delay.kind; sa.law.mu = h->delay.mu; sa.law.shift = h->delay.shift;
-  sa.seed = h->seed; sa.R = h->R; sa.replica_base = h->replica_base;
-  sa.j0 = h->n_updates; sa.iters = iters; sa.cap = h->cap; sa.K_stride = h->K_stride; sa.n_slots = h->n_slots;
-  sa.s = h->s; sa.tau = h->tau; sa.f = h->f; sa.wslot = h->wslot; sa.cur_slot = h->cur_slot;
-  sa.begin_slot = h->begin_slot; sa.clock = h->clock;
-  sa.t = h->tr.t; sa.K_used = h->tr.K_used; sa.worker = h->tr.worker; sa.stale = h->tr.stale; sa.seq = h->tr.seq;
-  sa.snap_slot = h->tr.snap_slot; sa.new_slot = h->tr.new_slot; sa.err = h->err;
-  // Loss-driven K: replicas pause where an update starts in a new interval and K may still grow; each
-  // round schedules every replica up to its next pause (or the target), runs the arithmetic that far,
-  // evaluates the full-data risk and sets the paused replicas' new K.  Rounds = interval crossings + 1.
-  const bool adaptive = h->ada_loss && h->t_interval > 0.0;
-  if (adaptive) {
-    if (!h->F0_ready) { if ((st = eval_into(h, h->F0)) != SIM_OK) return st; h->F0_ready = true; }
-    sa.adaptive = 1; sa.target = h->n_updates + iters; sa.done = h->done; sa.run_j0 = h->run_j0; sa.run_iters = h->run_iters;
-    sa.K_cur = h->K_cur; sa.q_last = h->q_last; sa.want_eval = h->want_eval;
+  // with a risk trace: stop at every multiple of eval_every and evaluate F(w_j) there (entry 0 is F(w_0))
+  const long long every = h->eval_every, need = 1 + (h->n_updates + iters) / every;
+  if (need > h->risk_cap) {
+    const long long nc = h->risk_cap * 2 > need ? h->risk_cap * 2 : need;
+    float* nb = nullptr;
+    CUDA_TRY(h, dev_alloc(&nb, (size_t)nc * h->R, h->stream, false));
+    if (h->risk && h->n_evals > 0)
+      CUDA_TRY(h, cudaMemcpyAsync(nb, h->risk, (size_t)h->n_evals * h->R * sizeof(float), cudaMemcpyDeviceToDevice, h->stream));
+    if (h->risk && !h->in_arena) { CUDA_TRY(h, cudaStreamSynchronize(h->stream)); cudaFree(h->risk); }
+    h->risk = nb; h->risk_cap = nc;
   }
-  for (long long round = 0;; ++round) {
-  CUDA_TRY(h, launch_schedule(sa, h->stream));
-
-  if (h->prob.model != SIM_NONE) {
-    NumericArgs a{};
-    if (adaptive) { a.run_j0 = h->run_j0; a.run_iters = h->run_iters; }
-    a.X = h->prob.X;
-    a.y = h->prob.model == SIM_LSQ ? static_cast<const void*>(h->prob.y) : static_cast<const void*>(h->prob.label);
-    a.w_ref = h->prob.w_ref; a.n = (uint64_t)h->prob.n; a.d = h->prob.d; a.m = h->m; a.model = (int)h->prob.model;
-    a.n_classes = h->prob.n_classes; a.eta = h->eta; a.seed = h->seed; a.replica_base = h->replica_base; a.R = h->R;
-    a.j0 = h->n_updates; a.iters = iters; a.cap = h->cap; a.K_stride = h->K_stride; a.is_async = h->is_async ? 1 : 0;
-    a.n_slots = h->n_slots; a.n_params = h->n_params; a.slot_stride = h->slot_stride;
-    a.K_used = h->tr.K_used; a.worker = h->tr.worker; a.seq = h->tr.seq; a.snap_slot = h->tr.snap_slot;
-    a.new_slot = h->tr.new_slot; a.begin_slot = h->begin_slot; a.loss = h->tr.loss; a.dist2 = h->tr.dist2;
-    a.w_state = h->w_state; a.pool = h->pool; a.err = h->err;
-    const char* why = nullptr;
-    cudaError_t ce = cudaSuccess;
-    switch (h->prob.model) {
-      case SIM_LSQ: case SIM_LOGISTIC: st = run_linear1(h, a); break;
-      case SIM_SOFTMAX:
-        ce = run_softmax_any(a, h->tune_stages, h->stream, &why);
-        st = why ? fail(h, SIM_ERR_ARG, why) : SIM_OK;
-        break;
-      case SIM_MLP2:
-        if (!h->mlp.Xq) {   // first run: bf16 copy of the data, per-update scratch, bf16 shadow of the initial W1
-          ce = mlp_scratch_alloc(h->mlp, h->prob.X, h->prob.n, h->prob.d, h->prob.hidden, h->prob.n_classes, h->m,
-                                 h->K_stride, h->R, h->n_slots, h->stream);
-          if (ce == cudaSuccess) ce = mlp_after_set_params(h->mlp, h->pool, h->slot_stride, h->stream);
-        }
-        if (ce == cudaSuccess) ce = run_mlp(a, h->mlp, h->mlp_maps, h->P, h->stream, &why);
-        if (ce == cudaSuccess && !h->is_async)   // synchronous variants ping-pong between two slots
-          ce = cudaMemsetAsync(h->cur_slot, (int)((h->n_updates + iters) & 1), (size_t)h->R, h->stream);
-        st = why ? fail(h, SIM_ERR_ARG, why) : SIM_OK;
-        break;
-      default: st = fail(h, SIM_ERR_ARG, "unknown model");
+  if (h->n_evals == 0) {
+    if ((st = eval_into(h, h->risk)) != SIM_OK) { h->poisoned = true; return st; }
+    h->n_evals = 1;
+  }
+  for (long long left = iters; left > 0;) {
+    const long long mark = (h->n_updates / every + 1) * every;
+    const long long seg = left < mark - h->n_updates ? left : mark - h->n_updates;
+    if ((st = run_span(h, seg)) != SIM_OK) return st;
+    left -= seg;
+    if (h->n_updates == mark) {
+      if ((st = eval_into(h, h->risk + (size_t)h->n_evals * h->R)) != SIM_OK) { h->poisoned = true; return st; }
+      ++h->n_evals;
     }
-    if (ce != cudaSuccess) st = fail(h, SIM_ERR_CUDA, std::string("numeric kernel launch: ") + cudaGetErrorString(ce));
-    if (st != SIM_OK) { h->poisoned = true; return st; }
   }
-  if (!adaptive) break;
-  if ((st = eval_into(h, h->Fcur)) != SIM_OK) { h->poisoned = true; return st; }
-  CUDA_TRY(h, cudaMemsetAsync(h->remaining, 0, sizeof(int), h->stream));
-  adasync_update_kernel<<<(h->R + 127) / 128, 128, 0, h->stream>>>(h->variant, h->P, h->K0, h->t_interval, h->R, sa.target, h->F0,
-                                                                  h->Fcur, h->clock, h->done, h->K_cur, h->q_last, h->want_eval,
-                                                                  h->remaining);
-  CUDA_TRY(h, cudaGetLastError());
-  int remaining = 0;
-  CUDA_TRY(h, cudaMemcpyAsync(&remaining, h->remaining, sizeof(int), cudaMemcpyDeviceToHost, h->stream));
-  CUDA_TRY(h, cudaStreamSynchronize(h->stream));
-  if (remaining == 0) break;
-  if (round > iters + 8) { h->poisoned = true; return fail(h, SIM_ERR_INTERNAL, "loss-driven K: no progress"); }
-  }
-  h->n_updates += iters;
   return SIM_OK;
 }
 
@@ -616,6 +728,7 @@ sim_status sim_set_adasync_loss(sim_handle* h, int32_t K0, double t_interval) {
   if (h->n_updates > 0 || h->cap > 0) return fail(h, SIM_ERR_STATE, "sim_set_adasync_loss is only allowed before sim_reserve / sim_run");
   if (!(t_interval > 0.0)) return fail(h, SIM_ERR_ARG, "t_interval must be > 0");
   if (K0 < 1 || K0 > h->P) return fail(h, SIM_ERR_ARG, "K0 must be in [1, P]");
+  if (h->eval_every > 0) return fail(h, SIM_ERR_STATE, "the loss-driven K rule cannot be combined with the risk trace (sim_set_eval_every)");
   const sim_model mdl = h->prob.model;
   if (mdl != SIM_LSQ && mdl != SIM_LOGISTIC && mdl != SIM_SOFTMAX)
     return fail(h, SIM_ERR_ARG, "the loss-driven K rule needs the full-data risk: LSQ, logistic or softmax");
@@ -644,6 +757,75 @@ sim_status sim_error_curve(const sim_handle* h, const double* grid, int32_t n_gr
   CUDA_TRY(h, cudaGetLastError());
   CUDA_TRY(h, cudaStreamSynchronize(h->stream));
   return SIM_OK;
+}
+
+sim_status sim_set_eval_every(sim_handle* h, int64_t every) {
+  if (!h) return fail(nullptr, SIM_ERR_ARG, "handle is NULL");
+  if (every < 0) return fail(h, SIM_ERR_ARG, "every must be >= 0");
+  if (h->n_updates > 0) return fail(h, SIM_ERR_STATE, "sim_set_eval_every is only allowed before the first sim_run");
+  if (every > 0 && h->prob.model == SIM_NONE) return fail(h, SIM_ERR_ARG, "a clock-only simulation has no risk to record");
+  if (every > 0 && h->ada_loss) return fail(h, SIM_ERR_STATE, "the risk trace cannot be combined with the loss-driven K rule");
+  h->eval_every = every;
+  return SIM_OK;
+}
+
+sim_status sim_risk_trace_size(const sim_handle* h, int64_t* n_evals) {
+  if (!h) return fail(nullptr, SIM_ERR_ARG, "handle is NULL");
+  if (n_evals) *n_evals = h->n_evals;
+  return SIM_OK;
+}
+
+sim_status sim_get_risk_trace(const sim_handle* h, float* risk, double* t) {
+  if (!h) return fail(nullptr, SIM_ERR_ARG, "handle is NULL");
+  sim_status st = device_error(h);
+  if (st != SIM_OK) return st;
+  if (h->n_evals == 0 || (!risk && !t)) return SIM_OK;
+  risk_trace_out_kernel<<<296, 256, 0, h->stream>>>(h->risk, h->tr.t, h->cap, h->eval_every, h->R, h->n_evals, risk, t);
+  CUDA_TRY(h, cudaGetLastError());
+  CUDA_TRY(h, cudaStreamSynchronize(h->stream));
+  return SIM_OK;
+}
+
+sim_status sim_risk_curve(const sim_handle* h, const double* grid, int32_t n_grid, float f_star, float* mean_err, int32_t* count) {
+  if (!h) return fail(nullptr, SIM_ERR_ARG, "handle is NULL");
+  if (!grid || !mean_err || !count || n_grid < 1) return fail(h, SIM_ERR_ARG, "grid, mean_err, count and n_grid >= 1 are required");
+  sim_status st = device_error(h);
+  if (st != SIM_OK) return st;
+  if (h->n_evals == 0) return fail(h, SIM_ERR_STATE, "no risk has been recorded (sim_set_eval_every, then sim_run)");
+  risk_curve_kernel<<<n_grid, 256, 0, h->stream>>>(h->risk, h->tr.t, h->cap, h->eval_every, h->R, h->n_evals, grid, f_star, mean_err, count);
+  CUDA_TRY(h, cudaGetLastError());
+  CUDA_TRY(h, cudaStreamSynchronize(h->stream));
+  return SIM_OK;
+}
+
+sim_status sim_risk_envelope(sim_handle* const* handles, int32_t n_handles, const double* grid, int32_t n_grid, float f_star,
+                             float* env, int32_t* best) {
+  if (!handles || n_handles < 1 || n_handles > 4096) return fail(nullptr, SIM_ERR_ARG, "sim_risk_envelope: handles and 1 <= n_handles <= 4096 are required");
+  if (!grid || !env || !best || n_grid < 1) return fail(nullptr, SIM_ERR_ARG, "sim_risk_envelope: grid, env, best and n_grid >= 1 are required");
+  for (int i = 0; i < n_handles; ++i)
+    if (!handles[i]) return fail(nullptr, SIM_ERR_ARG, "sim_risk_envelope: a handle is NULL");
+  float* curves = nullptr;
+  int* counts = nullptr;
+  const size_t cells = (size_t)n_handles * n_grid;
+  cudaError_t ce = cudaMalloc(&curves, cells * sizeof(float));
+  if (ce == cudaSuccess) ce = cudaMalloc(&counts, cells * sizeof(int));
+  sim_status st = ce == cudaSuccess ? SIM_OK : fail(nullptr, SIM_ERR_ALLOC, std::string("sim_risk_envelope: ") + cudaGetErrorString(ce));
+  std::string msg;
+  for (int i = 0; i < n_handles && st == SIM_OK; ++i) {      // each curve on its handle's stream; the call waits for it
+    st = sim_risk_curve(handles[i], grid, n_grid, f_star, curves + (size_t)i * n_grid, counts + (size_t)i * n_grid);
+    if (st != SIM_OK) msg = sim_last_error(handles[i]);
+  }
+  if (st == SIM_OK && msg.empty()) {
+    cudaStream_t stream = handles[0]->stream;
+    envelope_kernel<<<(n_grid + 127) / 128, 128, 0, stream>>>(curves, counts, n_handles, n_grid, env, best);
+    ce = cudaGetLastError();
+    if (ce == cudaSuccess) ce = cudaStreamSynchronize(stream);
+    if (ce != cudaSuccess) { st = SIM_ERR_CUDA; msg = cudaGetErrorString(ce); }
+  }
+  cudaFree(curves);
+  cudaFree(counts);
+  if (st != SIM_OK && !msg.empty()) return fail(nullptr, st, "sim_risk_envelope: " + msg);
+  return st;
 }
 
 sim_status sim_selftest_wait_timeout(sim_handle* h) {

@@ -262,3 +262,13 @@ def test_error_curve_by_hand():
     mean, cnt = error_curve(t, e, [0.25, 0.5, 1.0, 2.5, 3.0, 10.0])
     assert cnt.tolist() == [0, 1, 2, 2, 2, 2]
     assert mean.tolist() == [0.0, 20.0, 15.0, 14.0, 10.0, 5.0]
+
+
+def test_envelope_by_hand():
+    """Three curves on a grid of five points: the smallest value among the curves with data, lowest index on ties."""
+    from oracle.curves import envelope
+    curves = np.array([[9.0, 5.0, 4.0, 4.0, 1.0], [7.0, 6.0, 3.0, 4.0, 2.0], [1.0, 1.0, 8.0, 4.5, 0.5]])
+    counts = np.array([[0, 2, 2, 2, 2], [0, 1, 1, 1, 1], [0, 0, 3, 3, 3]])
+    env, best = envelope(curves, counts)
+    assert env.tolist() == [0.0, 5.0, 3.0, 4.0, 0.5]
+    assert best.tolist() == [-1, 0, 1, 0, 2]
