@@ -242,9 +242,42 @@ def entry(name, wl, variant, K_label, R, updates, ms, clocks, trace_K, peak, not
     return e
 
 
-def run_other_workloads(inputs, peak, local):
+def timed_eval(sim, local, reps=3):
+    """sim_eval_loss on the handle's current parameters: one warm-up call, then `reps` calls between two CUDA events."""
+    import torch
+    sim.eval_loss()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local, period=0.02)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        out = sim.eval_loss(to_numpy=False)
+    e1.record()
+    torch.cuda.synchronize()
+    assert bool(torch.isfinite(out).all())
+    return e0.elapsed_time(e1) / reps, sampler.finish()
+
+
+def run_other_workloads(inputs, peak, peaks, local, data2):
     import torch
     out = []
+    fp32_peak = 148 * 128 * 2 * 1.965e9 / 1e12       # TFLOP/s: 148 SMs x 128 FMA lanes x 2 flop at the 1965 MHz maximum clock
+
+    # -- full-data risk of all replicas (Eq. 1), K-sweep shape: one fp32 product X W^T over 1024 replicas
+    wl = inputs.WORKLOADS[2]
+    dev = device_data(data2)
+    sim = make_sim(wl, dev, "ksync", 8, wl.replicas)
+    sim.run(5)
+    ms, clocks = timed_eval(sim, local)
+    tf = 2.0 * wl.n * wl.d * wl.replicas / (ms * 1e-3) / 1e12
+    out.append({"workload": "full_data_risk_" + wl.name, "model": wl.model, "replicas": wl.replicas, "device_ms": ms,
+                "value": wl.replicas / (ms * 1e-3), "unit": "replica-evaluations/s", "clocks": clocks,
+                "roofline": {"bound": "alu", "achieved": tf, "peak": fp32_peak, "unit": "TFLOP/s", "frac": tf / fp32_peak,
+                             "note": "fp32 FMA product on the CUDA cores (the integer K of the loss-driven rule needs fp32 logits); "
+                                     "peak = 148 SMs x 128 lanes x 2 flop x 1965 MHz"}})
+    sim.close()
+    del dev
 
     def last_K(sim, updates):
         tr = sim.trace(to_numpy=False)
@@ -301,6 +334,13 @@ def run_other_workloads(inputs, peak, local):
     flops = 180 * wl.replicas * 4 * wl.m * (4 * wl.d * wl.hidden)      # forward and dW1 products, 2 flop per multiply-add
     e["tensor_tflops"] = flops / (ms * 1e-3) / 1e12
     out.append(e)
+    ms, clocks = timed_eval(sim, local, reps=2)
+    tf = 2.0 * wl.n * wl.d * wl.hidden * wl.replicas / (ms * 1e-3) / 1e12
+    tpeak = float(peaks.get("bf16_tflops", 1590.0))
+    out.append({"workload": "full_data_risk_" + wl.name, "model": wl.model, "replicas": wl.replicas, "device_ms": ms,
+                "value": wl.replicas / (ms * 1e-3), "unit": "replica-evaluations/s", "clocks": clocks,
+                "roofline": {"bound": "tensor", "achieved": tf, "peak": tpeak, "unit": "TFLOP/s", "frac": tf / tpeak,
+                             "note": "forward-only pass of the tcgen05 kernel over all 262144 rows for each of the 64 replicas"}})
     sim.close()
     del dev
     torch.cuda.empty_cache()
@@ -489,7 +529,7 @@ def main():
     torch.cuda.empty_cache()
 
     if world == 1 and not args.no_workloads:
-        line["workloads"] = run_other_workloads(inputs, peak, local)
+        line["workloads"] = run_other_workloads(inputs, peak, peaks, local, data)
 
     if not args.no_e2e:
         # the public one-shot call on pinned host buffers: one step's work (all 32 runs, U updates from

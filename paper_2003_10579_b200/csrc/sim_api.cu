@@ -12,6 +12,7 @@
 #include "linear_kernel.cuh"
 #include "softmax_kernel.cuh"
 #include "softmax_tm_kernel.cuh"
+#include "softmax_ws_kernel.cuh"
 #include "mlp_tc_kernel.cuh"
 #include "eval_kernel.cuh"
 

@@ -477,7 +477,7 @@ cudaError_t launch_softmax_tm(NumericArgs& a, cudaStream_t stream) {
   return cudaGetLastError();
 }
 
-inline cudaError_t run_softmax_any(NumericArgs& a, int tune_stages, cudaStream_t stream, const char** why) {
+inline cudaError_t run_softmax_tm_any(NumericArgs& a, int tune_stages, cudaStream_t stream, const char** why) {
   *why = nullptr;
   if (softmax_tm_supported(a.d, a.n_classes, a.m)) {
     const int kp = (a.d / 2 + 128 * SMX_TM_NG - 1) / (128 * SMX_TM_NG);
