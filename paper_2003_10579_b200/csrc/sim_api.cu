@@ -11,7 +11,6 @@
 
 #include "linear_kernel.cuh"
 #include "softmax_kernel.cuh"
-#include "softmax_tm_kernel.cuh"
 #include "softmax_ws_kernel.cuh"
 #include "mlp_tc_kernel.cuh"
 #include "eval_kernel.cuh"

@@ -2,9 +2,23 @@
 // warps do nothing but the two FMA passes; a fourth warpgroup stages rows (one warp) and forms the
 // softmax terms (three warps), on a small share of the registers.
 //
-// The parameters live in tensor memory and the gradient accumulator in registers exactly as in
-// softmax_tm_kernel (thread t of the 384 owns feature pairs t + 384 k; tensor-memory lane t mod 128
-// holds the columns of its three owners).  What differs is who waits for whom.  This path is
+// Ownership.  The d/2 pairs of adjacent features are dealt to the 384 FMA threads: thread t owns pairs
+// t + 384 k (k < KP).  For its pairs and all classes it keeps the gradient accumulator G in registers
+// for the whole update and the parameters W_tau in 20 KP columns of its own tensor-memory lane
+// (lane t mod 128, columns 20 KP (t / 128) ...; column 20 k + 2 c + h holds W[c][feature h of pair k]):
+// tensor memory serves as a 120 KB register-file extension with its own read path, no MMA is issued.
+// The update W <- W - (eta / (K m)) G (Eq. 2 / Eq. 3) is thread-local: tcgen05.ld, FMA, tcgen05.st.
+// Per tile:
+//   logits    Z = X_tile W_tau^T.  The three groups of four warps take different rows (TG each); thread
+//             (lane L of the 128, group g) walks the whole of tensor-memory lane L - the columns of all
+//             three owners.  One warp transposition reduce and a four-way sum finish the logits.
+//   softmax   D = softmax(Z) - onehot(label), loss: 16 lanes per row.
+//   gradient  G += D^T X_tile: every FMA thread, every row, own pairs, packed fp32x2 FMAs (the two
+//             features of a pair), for nine of the ten class slots - the rows of D sum to zero, so the
+//             tenth slot's gradient is minus the sum of the others and is formed once per update.
+// Plain fp32 FMAs: the 1e-5 parity bound on the parameters rules out reduced-precision tensor-core operands.
+//
+// Who waits for whom.  This path is
 // bound by instruction issue (20 FMA per 4-byte feature, every other instruction costs an FMA
 // slot), and in a kernel where all warps walk through "logits, barrier, softmax, barrier,
 // gradient" together the FMA pipe idles while a few lanes form the softmax terms and while one
@@ -28,7 +42,7 @@
 // a bounded poll of an mbarrier; a wait that runs out raises a flag in shared memory that ends all
 // other waits early, and the error word is set.
 #pragma once
-#include "softmax_tm_kernel.cuh"
+#include "tmem_util.cuh"
 
 namespace ssim {
 
@@ -266,9 +280,14 @@ __global__ void __launch_bounds__(SWS_THREADS, 1) softmax_ws_kernel(NumericArgs 
       return ok;
     };
 
-    uint64_t G[CP][KP];      // the two features of a pair
+    // Gradient accumulator of the first nine class slots only.  The rows of D = softmax(Z) - onehot sum to zero over the
+    // classes, hence so do the rows of the gradient D^T X: the tenth slot is minus the sum of the other nine, formed
+    // once per update instead of being accumulated with a tenth of the gradient pass's FMAs (with fewer than ten classes
+    // the tenth slot is padding and its gradient is zero).
+    constexpr int GC = CP - 1;
+    uint64_t G[GC][KP];      // the two features of a pair
 #pragma unroll
-    for (int c = 0; c < CP; ++c)
+    for (int c = 0; c < GC; ++c)
 #pragma unroll
       for (int k = 0; k < KP; ++k) G[c][k] = 0ull;
     long long j = my_j0;
@@ -292,12 +311,9 @@ __global__ void __launch_bounds__(SWS_THREADS, 1) softmax_ws_kernel(NumericArgs 
           const float4 v = reinterpret_cast<const float4*>(delta)[q * (SMT_DSTR / 4) + c4];
           dv[4 * c4] = v.x; dv[4 * c4 + 1] = v.y; dv[4 * c4 + 2] = v.z; dv[4 * c4 + 3] = v.w;
         }
-        {
-          const float2 v = reinterpret_cast<const float2*>(delta)[q * (SMT_DSTR / 2) + 4];
-          dv[8] = v.x; dv[9] = v.y;
-        }
+        dv[8] = delta[q * SMT_DSTR + 8];
 #pragma unroll
-        for (int c = 0; c < CP; ++c) {
+        for (int c = 0; c < GC; ++c) {
           const uint64_t dd = pack2(dv[c], dv[c]);
 #pragma unroll
           for (int k = 0; k < KP; ++k) G[c][k] = ffma2(dd, x2[k], G[c][k]);
@@ -333,10 +349,11 @@ __global__ void __launch_bounds__(SWS_THREADS, 1) softmax_ws_kernel(NumericArgs 
           for (int s = 0; s < TG; ++s) x[s] = rowp[s * NG * (DS / 2) + 128 * gp + NT * k];
           tm_wait_ld();
 #pragma unroll
-          for (int s = 0; s < TG; ++s)
+          for (int s = 0; s < TG; ++s) {
 #pragma unroll
             for (int c = 0; c < CP; ++c)
               acc[s * CP + c] = fmaf(x[s].y, w[2 * c + 1], fmaf(x[s].x, w[2 * c], acc[s * CP + c]));
+          }
         }
         tm_reduce_steps<16, NV>(acc, lane);
         if (red_idx >= 0) red_s[(buf * NW + warp) * 32 + red_idx] = acc[0];
@@ -372,11 +389,18 @@ __global__ void __launch_bounds__(SWS_THREADS, 1) softmax_ws_kernel(NumericArgs 
             const int p = tid + NT * k;
             float w[WC];
             if (!ASYNC) { tm_ld20(t_own + k * WC, w); tm_wait_ld(); }
+            float s0 = 0.f, s1 = 0.f;      // sum of the nine accumulated slots, in slot order
 #pragma unroll
             for (int c = 0; c < CP; ++c) {
               float g0, g1;
-              unpack2(G[c][k], g0, g1);
-              G[c][k] = 0ull;
+              if (c < GC) {
+                unpack2(G[c][k], g0, g1);
+                G[c][k] = 0ull;
+                s0 += g0; s1 += g1;
+              } else {
+                g0 = C == CP ? -s0 : 0.f;
+                g1 = C == CP ? -s1 : 0.f;
+              }
               if (ASYNC) {
                 if (p < dp && c < C) {
                   float2 v = reinterpret_cast<const float2*>(w_from + (size_t)c * d)[p];
@@ -497,9 +521,10 @@ inline cudaError_t run_softmax_any(NumericArgs& a, int tune_stages, cudaStream_t
       case 3: e = launch_softmax_ws<3>(a, stream, &fits); break;
       default: e = launch_softmax_ws<4>(a, stream, &fits); break;
     }
-    if (fits || e != cudaSuccess) return e;
+    if (!fits) *why = "softmax: the kernel was built with fewer registers per thread than its register split needs";
+    return e;
   }
-  return run_softmax_tm_any(a, tune_stages, stream, why);
+  return run_softmax(a, tune_stages, stream, why);
 }
 
 }  // namespace ssim
