@@ -268,14 +268,17 @@ __global__ void __launch_bounds__(NT) linear1_kernel(NumericArgs a) {
   int st = 0;             // stage and phase parity of tile `it`, kept as counters (it % S and it / S are 64-bit divisions)
   uint32_t parity = 0;
   for (long long it = 0;; ++it, parity ^= (uint32_t)(st + 1 == S), st = (st + 1 == S ? 0 : st + 1)) {
-    // A wait that runs out does not leave on its own: the thread goes on to the tile's block barrier (on whatever the
-    // stage holds - shared memory only, no access depends on it) and the whole block votes there, so that either
-    // every thread of the block drains or none does.
-    const bool ok = mbar_wait(smem_addr(&full[st]), parity);
+    // A thread whose wait runs out does not leave: the others may already be on their way to the tile's block barrier.
+    // It stops waiting for good and follows the block through the rest of the run in step - same barriers, arithmetic on
+    // whatever the stages hold - and reports at the end.  The control flow cannot split: it is steered by the tile's
+    // descriptor, which the producer wrote at least one block barrier before any thread reads it, whether or not the
+    // tile's copies ever land; so all threads of the block take the same branches by construction.
+    const bool ok = !failed && mbar_wait(smem_addr(&full[st]), parity);
+    failed = failed || !ok;
     const TileInfo ti = info_s[st];
     const float* tile = rows_s + (size_t)st * T * d;
 
-    if (ASYNC && ok && (ti.flags & TILE_FIRST_OF_TASK)) {
+    if (ASYNC && (ti.flags & TILE_FIRST_OF_TASK)) {
       if (ti.snap == cur_slot) {
 #pragma unroll
         for (int e = 0; e < E; ++e) w_tau[e] = w_cur[e];
@@ -325,7 +328,7 @@ __global__ void __launch_bounds__(NT) linear1_kernel(NumericArgs a) {
 #pragma unroll
       for (int q = 0; q < T; ++q) red_s[((it & 1) * NW + warp) * T + q] = part[q];
     }
-    if (__syncthreads_or(!ok)) { failed = true; break; }
+    __syncthreads();
     // every thread is past its reads of the previous tile's stage: refill it
     if (warp == 0) issue_tile(it + S - 1);
 
