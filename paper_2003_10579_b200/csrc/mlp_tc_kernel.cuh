@@ -86,24 +86,27 @@ struct TcLayout {   // shared-memory plan of the forward kernel (offsets from a 
 };
 // The operands have rings of their own: A (128 samples x 64 k, 16 KB) in `sa` slots; B in `sb` slots of
 // [n_inst x 64 k], n_inst = H (H <= 256) or H/2 - half a k-block of W1 per slot, so that several loads of
-// 32 KB are in flight instead of one of 64 KB.
+// 32 KB are in flight instead of one of 64 KB.  The main loop is bound by the latency of those loads, i.e. by the bytes
+// in flight, so everything the epilogue alone needs (W2 padded to 16 classes, the partial logits) lives in the A ring's
+// bytes, which are free once the last MMA has completed, and the B ring gets the room.
 inline __host__ __device__ TcLayout tc_forward_layout(int H) {
   TcLayout L;
   L.b_bytes = (H > 256 ? H / 2 : H) * 128;
   L.sa = 4;
-  L.sb = 3;
+  L.sb = 4;
+  L.off_w2 = 0;                                   // [H][16] floats, after the main loop
+  L.off_zx = L.off_w2 + H * 16 * 4;               // partial logits of the two column halves: [2][128][16], after the main loop
   L.off_b = L.sa * TC_A_BYTES;
-  L.off_w2 = L.off_b + L.sb * L.b_bytes;
-  L.off_b1 = L.off_w2 + H * 16 * 4;
+  L.off_b1 = L.off_b + L.sb * L.b_bytes;
   L.off_b2 = L.off_b1 + H * 4;
   L.off_rows = L.off_b2 + 64;
   L.off_labels = L.off_rows + 128 * 4;
-  L.off_zx = L.off_labels + 128 * 4;              // partial logits of the two column halves: [2][128][16]
-  L.off_bars = L.off_zx + 2 * 128 * 16 * 4;
+  L.off_bars = L.off_labels + 128 * 4;
   L.off_tmem = L.off_bars + 8 * (2 * L.sa + 2 * L.sb + 1);
   L.total = L.off_tmem + 16 + 1024;   // slack for the manual 1024-byte alignment
   return L;
 }
+static_assert(512 * 16 * 4 + 2 * 128 * 16 * 4 <= 4 * TC_A_BYTES, "W2 and the partial logits must fit the A ring's bytes");
 
 // EVAL = true is the forward-only form for the full-data risk F(w) of Eq. 1: one CTA per (replica, 128 consecutive rows
 // of the data set), the replica's current version, and only the rows' losses leave the CTA.
@@ -240,18 +243,26 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmW, MlpArgs g) {
     const size_t grow = task * m + (size_t)mt * 128 + row;
     const int part = mt * 4 + q, parts = mtiles * 4;
     if (ehalf) {
-      // ---- helpers, during the main loop: b1, W2 (rows padded to 16 classes) and b2 of the snapshot ----
+      // ---- helpers: b1 and b2 of the snapshot during the main loop; W2 (rows padded to 16 classes) goes into the A
+      //      ring's bytes once the last MMA has read them (its values wait in registers meanwhile) ----
       const int t = tid - 192;
       const float* b1 = wsnap + dH;
       const float* W2 = b1 + H;
       const float* b2 = W2 + (size_t)H * C;
-#pragma unroll 8
-      for (int i = t; i < H * 16; i += 128) {
-        const int col = i >> 4, c = i & 15;
-        W2_s[i] = c < C ? W2[(size_t)col * C + c] : 0.f;
-      }
       for (int i = t; i < H; i += 128) b1_s[i] = b1[i];
       if (t < 16) b2_s[t] = t < C ? b2[t] : 0.f;
+      float w2v[64];                                 // H * 16 / 128 <= 64 entries per thread
+#pragma unroll
+      for (int u = 0; u < 64; ++u) {
+        const int i = t + 128 * u, col = i >> 4, c = i & 15;
+        w2v[u] = (i < H * 16 && c < C) ? W2[(size_t)col * C + c] : 0.f;
+      }
+      if (!mbar_wait(acc_bar, 0)) failed = true;
+#pragma unroll
+      for (int u = 0; u < 64; ++u) {
+        const int i = t + 128 * u;
+        if (i < H * 16) W2_s[i] = w2v[u];
+      }
     } else
     // ---- A producer: thread t copies 16-byte piece (t & 7) of rows (t >> 3) + 16 i, i < 8.  A k-block is
     //      signalled FWD_LAG k-blocks after it was issued; the ring is deeper than that (SA > FWD_LAG + 1), so
