@@ -964,6 +964,7 @@ sim_status sim_sweep_host(const sim_problem* problem, int32_t P, int32_t n_runs,
   const size_t RJ = (size_t)n_replicas * (size_t)iters;
   DeviceArena arena;                    // the runs' state, parameters and traces: a few chunks instead of hundreds of buffers
   t_arena = &arena;
+  cudaEvent_t uploaded = nullptr;
   do {
     void *X, *y, *lab, *wr, *dw0;
     if (!up(problem->X, (size_t)dp.n * dp.d * 4, &X)) break;
@@ -972,10 +973,15 @@ sim_status sim_sweep_host(const sim_problem* problem, int32_t P, int32_t n_runs,
     if (!up(problem->w_ref, (size_t)np * 4, &wr)) break;
     if (!up(w0, (size_t)np * 4, &dw0)) break;
     dp.X = (const float*)X; dp.y = (const float*)y; dp.label = (const int32_t*)lab; dp.w_ref = (const float*)wr;
-    if (cudaDeviceSynchronize() != cudaSuccess) { st = SIM_ERR_CUDA; msg = "upload failed"; break; }
+    // the copies above are in flight on the default stream; the runs' streams wait for them on the device, so that the host
+    // sets the runs up meanwhile
+    if (cudaEventCreateWithFlags(&uploaded, cudaEventDisableTiming) != cudaSuccess || cudaEventRecord(uploaded, nullptr) != cudaSuccess) {
+      st = SIM_ERR_CUDA; msg = "upload failed"; break;
+    }
     // every run gets its own stream: the runs are independent and overlap on the device
     for (int i = 0; i < n_runs && st == SIM_OK; ++i) {
-      if (cudaStreamCreateWithFlags(&streams[i], cudaStreamNonBlocking) != cudaSuccess) { st = SIM_ERR_CUDA; msg = "stream creation failed"; break; }
+      if (cudaStreamCreateWithFlags(&streams[i], cudaStreamNonBlocking) != cudaSuccess ||
+          cudaStreamWaitEvent(streams[i], uploaded, 0) != cudaSuccess) { st = SIM_ERR_CUDA; msg = "stream creation failed"; break; }
       st = sim_create(&dp, P, Ks[i], (sim_variant)variants[i], delay, eta, m, seed, n_replicas, replica_base, streams[i], &hs[i]);
       if (st != SIM_OK) { msg = g_last_error; break; }
       if ((st = sim_reserve(hs[i], iters)) != SIM_OK) { msg = sim_last_error(hs[i]); break; }
@@ -1002,6 +1008,7 @@ sim_status sim_sweep_host(const sim_problem* problem, int32_t P, int32_t n_runs,
   }
   t_arena = nullptr;
   cudaDeviceSynchronize();
+  if (uploaded) cudaEventDestroy(uploaded);
   arena.release();
   for (void* p : owned) cudaFree(p);
   if (st != SIM_OK) return fail(nullptr, st, "sim_sweep_host: " + msg);
