@@ -3,9 +3,9 @@
 // curves and behind the rule that raises K in Algorithm 1.
 //
 // The logits of all replicas are one dense product Z = X W^T (n x d times d x (R*C)), so the data
-// set is read once per 64 (replica, class) columns instead of once per replica.  fp32 FMAs
+// set is read once per 128 (replica, class) columns instead of once per replica.  fp32 FMAs
 // (a loss at its noise floor needs the full fp32 mantissa of the logits, so no tf32 / bf16 tensor
-// path), classic shared-memory tiling: block = 128 rows x 64 columns, 256 threads x (8 x 4).
+// path), shared-memory tiling: block = 128 rows x 128 columns, 256 threads x (8 x 8).
 // The per-sample losses are summed in fp64 in a fixed order (warp tree, then row blocks in
 // sequence in a second kernel): the result does not vary from run to run.
 #pragma once
@@ -13,20 +13,25 @@
 
 namespace ssim {
 
-constexpr int EV_BM = 128, EV_BN = 64, EV_BK = 16;
+constexpr int EV_BM = 128, EV_BN = 128, EV_BK = 16;
+constexpr int EV_LDA = EV_BM + 4, EV_LDB = EV_BN + 4;   // padded leading dimensions of the operand tiles [k][row], [k][column]
+constexpr int EV_OPERAND_FLOATS = 2 * EV_BK * (EV_LDA + EV_LDB);   // A and B, two buffers each
+constexpr int EV_CG = EV_BN / 64;                       // groups of four columns per thread
+constexpr int EV_Z_FLOATS = EV_BM * (EV_BN + 1);
+constexpr size_t EV_SMEM_BYTES = sizeof(float) * (EV_Z_FLOATS > EV_OPERAND_FLOATS ? EV_Z_FLOATS : EV_OPERAND_FLOATS);
 
 struct EvalArgs {
   const float* X;
   const void* y;
   long long n;
   int d, C, model, R;
-  int RB;                       // replicas per column block: floor(64 / C)
+  int RB;                       // replicas per column block: floor(EV_BN / C)
   const float* w_state;         // [R][n_params] or null
   const float* pool;            // [R][n_slots][slot_stride] or null
   const uint8_t* cur_slot;      // [R] (pool)
   int n_slots;
   long long n_params, slot_stride;
-  double* partial;              // [row_blocks][R]
+  double* partial;              // [row blocks][R]
   int row_blocks;
   float* out;                   // [R]
 };
@@ -36,61 +41,111 @@ __device__ __forceinline__ const float* eval_params(const EvalArgs& a, int r) {
   return a.w_state + (size_t)r * a.n_params;
 }
 
-__global__ void __launch_bounds__(256) eval_loss_kernel(EvalArgs a) {
-  __shared__ float As[EV_BK][EV_BM + 4];
-  __shared__ float Bs[EV_BK][EV_BN + 4];
-  __shared__ float Zs[EV_BM][EV_BN + 1];
+// Block = 128 rows x 128 (replica, class) columns, 256 threads x (8 x 8) accumulators, two blocks per SM.  (At 128 B/clk
+// of shared-memory return bandwidth against 128 FMA/clk an 8 x 8 register tile needs one byte per FMA, so the two pipes
+// are about equally loaded; 8 x 16 tiles at one block per SM need 0.75 but were slower: 41 against 44 TFLOP/s, the
+// second block's warps hide more than the saved loads buy.)  Both operands are stored with k
+// contiguous (rows of X, rows of W), so a tile is read as float4s along k into registers and written transposed into
+// shared memory ([k][row], [k][column]); the next tile's global loads are in flight while the current one is multiplied
+// (register prefetch, two shared-memory buffers, one block barrier per k-tile).  A thread's eight rows and eight columns
+// are groups of four, 64 apart, so that its float4 reads of a k-row are conflict-free.  After the k loop the logits go
+// to shared memory (over the operand buffers) and the per-sample losses are formed and summed as before.
+__global__ void __launch_bounds__(256, 2) eval_loss_kernel(EvalArgs a) {
+  extern __shared__ __align__(16) float ev_smem[];
   __shared__ double sums_s[EV_BN][4];
+  float* As = ev_smem;                                   // [2][EV_BK][EV_LDA]
+  float* Bs = ev_smem + 2 * EV_BK * EV_LDA;              // [2][EV_BK][EV_LDB]
+  float* Zs = ev_smem;                                   // [EV_BM][EV_BN + 1], after the k loop
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   const long long row0 = (long long)blockIdx.x * EV_BM;
   const int rep0 = blockIdx.y * a.RB;
   const int d = a.d, C = a.C;
 
-  // B operand: column c of the block = (replica rep0 + c / C, class c % C)
-  const int bcol = tid >> 2, bkq = tid & 3;
-  const int brep = rep0 + bcol / C, bcls = bcol % C;
-  const bool bvalid = bcol < a.RB * C && brep < a.R;
-  const float* bptr = bvalid ? eval_params(a, brep) + (size_t)bcls * d : nullptr;
-
-  float acc[8][4];
+  // global -> register mapping of a tile: thread takes k-quad kq of rows lr, lr + 64 and columns lr + 64 i, i < EV_CG
+  const int lr = tid >> 2, kq = tid & 3;
+  const float* aptr[2];
+  const float* bptr[EV_CG];
 #pragma unroll
-  for (int i = 0; i < 8; ++i)
-#pragma unroll
-    for (int jn = 0; jn < 4; ++jn) acc[i][jn] = 0.f;
-
-  for (int k0 = 0; k0 < d; k0 += EV_BK) {
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      const int row = (tid >> 2) + 64 * i, kq = tid & 3;
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (row0 + row < a.n && k0 + 4 * kq < d) v = *reinterpret_cast<const float4*>(a.X + (size_t)(row0 + row) * d + k0 + 4 * kq);
-      As[4 * kq][row] = v.x; As[4 * kq + 1][row] = v.y; As[4 * kq + 2][row] = v.z; As[4 * kq + 3][row] = v.w;
-    }
-    {
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (bvalid && k0 + 4 * bkq < d) v = *reinterpret_cast<const float4*>(bptr + k0 + 4 * bkq);
-      Bs[4 * bkq][bcol] = v.x; Bs[4 * bkq + 1][bcol] = v.y; Bs[4 * bkq + 2][bcol] = v.z; Bs[4 * bkq + 3][bcol] = v.w;
-    }
-    __syncthreads();
-#pragma unroll
-    for (int k = 0; k < EV_BK; ++k) {
-      float av[8], bv[4];
-      const float4 a0 = *reinterpret_cast<const float4*>(&As[k][ty * 8]);
-      const float4 a1 = *reinterpret_cast<const float4*>(&As[k][ty * 8 + 4]);
-      const float4 b0 = *reinterpret_cast<const float4*>(&Bs[k][tx * 4]);
-      av[0] = a0.x; av[1] = a0.y; av[2] = a0.z; av[3] = a0.w; av[4] = a1.x; av[5] = a1.y; av[6] = a1.z; av[7] = a1.w;
-      bv[0] = b0.x; bv[1] = b0.y; bv[2] = b0.z; bv[3] = b0.w;
-#pragma unroll
-      for (int i = 0; i < 8; ++i)
-#pragma unroll
-        for (int jn = 0; jn < 4; ++jn) acc[i][jn] = fmaf(av[i], bv[jn], acc[i][jn]);
-    }
-    __syncthreads();
+  for (int i = 0; i < 2; ++i) {
+    const long long row = row0 + lr + 64 * i;
+    aptr[i] = row < a.n ? a.X + (size_t)row * d : nullptr;
   }
 #pragma unroll
+  for (int i = 0; i < EV_CG; ++i) {
+    const int col = lr + 64 * i;                         // column of the block = (replica rep0 + col / C, class col % C)
+    const int rep = rep0 + col / C;
+    bptr[i] = (col < a.RB * C && rep < a.R) ? eval_params(a, rep) + (size_t)(col % C) * d : nullptr;
+  }
+  auto fetch = [&](int k0, float4 (&av)[2], float4 (&bv)[EV_CG]) {
+    const bool in = k0 + 4 * kq < d;                     // d is a multiple of 4: a quad is inside or outside
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      av[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (in && aptr[i]) av[i] = *reinterpret_cast<const float4*>(aptr[i] + k0 + 4 * kq);
+    }
+#pragma unroll
+    for (int i = 0; i < EV_CG; ++i) {
+      bv[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (in && bptr[i]) bv[i] = *reinterpret_cast<const float4*>(bptr[i] + k0 + 4 * kq);
+    }
+  };
+  auto stash = [&](int buf, const float4 (&av)[2], const float4 (&bv)[EV_CG]) {
+    float* A_ = As + buf * EV_BK * EV_LDA;
+    float* B_ = Bs + buf * EV_BK * EV_LDB;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const int rc = lr + 64 * i;
+      A_[(4 * kq) * EV_LDA + rc] = av[i].x; A_[(4 * kq + 1) * EV_LDA + rc] = av[i].y;
+      A_[(4 * kq + 2) * EV_LDA + rc] = av[i].z; A_[(4 * kq + 3) * EV_LDA + rc] = av[i].w;
+    }
+#pragma unroll
+    for (int i = 0; i < EV_CG; ++i) {
+      const int rc = lr + 64 * i;
+      B_[(4 * kq) * EV_LDB + rc] = bv[i].x; B_[(4 * kq + 1) * EV_LDB + rc] = bv[i].y;
+      B_[(4 * kq + 2) * EV_LDB + rc] = bv[i].z; B_[(4 * kq + 3) * EV_LDB + rc] = bv[i].w;
+    }
+  };
+
+  float acc[8][4 * EV_CG];
+#pragma unroll
   for (int i = 0; i < 8; ++i)
 #pragma unroll
-    for (int jn = 0; jn < 4; ++jn) Zs[ty * 8 + i][tx * 4 + jn] = acc[i][jn];
+    for (int jn = 0; jn < 4 * EV_CG; ++jn) acc[i][jn] = 0.f;
+
+  float4 av[2], bv[EV_CG];
+  fetch(0, av, bv);
+  stash(0, av, bv);
+  __syncthreads();
+  const int n_tiles = (d + EV_BK - 1) / EV_BK;
+  for (int kt = 0; kt < n_tiles; ++kt) {
+    const int buf = kt & 1;
+    if (kt + 1 < n_tiles) fetch((kt + 1) * EV_BK, av, bv);
+    const float* A_ = As + buf * EV_BK * EV_LDA;
+    const float* B_ = Bs + buf * EV_BK * EV_LDB;
+#pragma unroll
+    for (int k = 0; k < EV_BK; ++k) {
+      const float4 a0 = *reinterpret_cast<const float4*>(A_ + k * EV_LDA + ty * 4);
+      const float4 a1 = *reinterpret_cast<const float4*>(A_ + k * EV_LDA + 64 + ty * 4);
+      const float ar[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+#pragma unroll
+      for (int g = 0; g < EV_CG; ++g) {
+        const float4 b = *reinterpret_cast<const float4*>(B_ + k * EV_LDB + 64 * g + tx * 4);
+        const float br[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+#pragma unroll
+          for (int jn = 0; jn < 4; ++jn) acc[i][4 * g + jn] = fmaf(ar[i], br[jn], acc[i][4 * g + jn]);
+      }
+    }
+    if (kt + 1 < n_tiles) stash(buf ^ 1, av, bv);
+    __syncthreads();
+  }
+  // logits to shared memory (the operand buffers are free after the last barrier)
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int jn = 0; jn < 4 * EV_CG; ++jn)
+      Zs[((i >> 2) * 64 + ty * 4 + (i & 3)) * (EV_BN + 1) + (jn >> 2) * 64 + tx * 4 + (jn & 3)] = acc[i][jn];
   __syncthreads();
 
   // per-sample losses: pair p = (replica rr, row): consecutive threads take consecutive rows
@@ -99,7 +154,7 @@ __global__ void __launch_bounds__(256) eval_loss_kernel(EvalArgs a) {
     const int rr = p / EV_BM, row = p % EV_BM;
     double f = 0.0;
     if (row0 + row < a.n && rep0 + rr < a.R) {
-      const float* z = &Zs[row][rr * C];
+      const float* z = &Zs[row * (EV_BN + 1) + rr * C];
       if (a.model == M_LSQ) {
         const float res = z[0] - reinterpret_cast<const float*>(a.y)[row0 + row];
         f = 0.5 * (double)res * (double)res;

@@ -341,7 +341,8 @@ sim_status eval_into(sim_handle* h, float* loss) {
   if (!h->eval_partial) CUDA_TRY(h, dev_alloc(&h->eval_partial, (size_t)e.row_blocks * h->R, h->stream, false));
   e.partial = h->eval_partial; e.out = loss;
   dim3 grid((unsigned)e.row_blocks, (unsigned)((h->R + e.RB - 1) / e.RB));
-  eval_loss_kernel<<<grid, 256, 0, h->stream>>>(e);
+  CUDA_TRY(h, cudaFuncSetAttribute(eval_loss_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)EV_SMEM_BYTES));
+  eval_loss_kernel<<<grid, 256, EV_SMEM_BYTES, h->stream>>>(e);
   CUDA_TRY(h, cudaGetLastError());
   eval_loss_finish_kernel<<<(h->R + 127) / 128, 128, 0, h->stream>>>(e);
   CUDA_TRY(h, cudaGetLastError());
