@@ -211,12 +211,14 @@ __global__ void __launch_bounds__(NT) linear1_kernel(NumericArgs a) {
     for (int e = 0; e < E; ++e) { g[e] = 0.f; w_tau[e] = w_cur[e]; }
   }
 
-  // ---- producer (warp 0): stage tiles of rows ahead of the arithmetic ----
+  // ---- producer (the last warp; thread 0 of the first records losses and distances): stage tiles of rows ahead of the
+  //      arithmetic.  For the narrowest rows the block has one warp more than the columns need, so that drawing indices
+  //      and issuing copies overlaps the arithmetic instead of taking turns with it ----
   ScheduleWalk walk;
   walk.done = true;
   int prod_st = 0;
   auto issue_tile = [&](long long) {
-    // called by all lanes of warp 0; the stage's previous contents have been consumed
+    // called by all lanes of the producer warp; the stage's previous contents have been consumed
     if (walk.done) return;
     const int st = prod_st;   // tiles are issued in order: a counter, not a 64-bit modulo per tile
     if (++prod_st == S) prod_st = 0;
@@ -254,7 +256,7 @@ __global__ void __launch_bounds__(NT) linear1_kernel(NumericArgs a) {
     }
     walk.advance(a);
   };
-  if (warp == 0) {
+  if (warp == NW - 1) {
     walk.start(a, r, my_j0, my_iters);
     walk.tiles_per_task = (m + T - 1) / T;
     for (int s = 0; s < S - 1; ++s) issue_tile(s);
@@ -330,7 +332,7 @@ __global__ void __launch_bounds__(NT) linear1_kernel(NumericArgs a) {
     }
     __syncthreads();
     // every thread is past its reads of the previous tile's stage: refill it
-    if (warp == 0) issue_tile(it + S - 1);
+    if (warp == NW - 1) issue_tile(it + S - 1);
 
     // ---- a_q = dl/dz and the loss ----
     float aq[T], zq[T];

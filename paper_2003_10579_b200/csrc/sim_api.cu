@@ -246,7 +246,9 @@ sim_status launch_linear1(sim_handle* h, NumericArgs& a) {
 
 sim_status run_linear1(sim_handle* h, NumericArgs& a) {
   const int d4 = a.d / 4;
-  if (d4 <= 32) return launch_linear1<32, 1, 8>(h, a);
+  // up to 32 column chunks: with few replicas (at most two per SM the run is a chain of latencies) a second warp that only
+  // produces overlaps drawing indices and issuing copies with the arithmetic; with many, one warp per replica packs better
+  if (d4 <= 32 && a.R > 296) return launch_linear1<32, 1, 8>(h, a);
   if (d4 <= 64) return launch_linear1<64, 1, 8>(h, a);
   if (d4 <= 128) return launch_linear1<128, 1, 4>(h, a);
   if (d4 <= 256) {
@@ -269,8 +271,7 @@ sim_status run_linear1(sim_handle* h, NumericArgs& a) {
 size_t linear1_min_smem(int d, int m, int R) {
   const int d4 = d / 4;
   int NT = 512, T = 2;
-  if (d4 <= 32) { NT = 32; T = 8; }
-  else if (d4 <= 64) { NT = 64; T = 8; }
+  if (d4 <= 64) { NT = 64; T = 8; }       // (a block of 32 threads needs no more)
   else if (d4 <= 128) { NT = 128; T = 4; }
   else if (d4 <= 256) { NT = 128; T = 4; }
   else if (d4 <= 512) { NT = 256; T = 4; }
