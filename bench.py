@@ -158,6 +158,13 @@ def oracle_all_cores(reps, updates, max_procs=32):
     return done, dt, n
 
 
+def headline_config(wl, R, U):
+    """The `config` object of the headline workload: the same for both arms."""
+    return {"workload": wl.name, "n": wl.n, "d": wl.d, "P": wl.P, "m": wl.m, "runs": len(wl.runs),
+            "replicas_per_run_per_gpu": R, "updates_per_step": U,
+            "l2": "input X is 256 MiB, larger than L2; rows are gathered at random"}
+
+
 def run_reference(args, wl):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -177,7 +184,7 @@ def run_reference(args, wl):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "n": wl.n, "d": wl.d, "P": wl.P, "m": wl.m, "runs": len(wl.runs)},
+        "config": headline_config(wl, args.replicas or wl.replicas, args.updates_per_step),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -522,9 +529,7 @@ def main():
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": wl.name, "n": wl.n, "d": wl.d, "P": wl.P, "m": wl.m, "runs": len(wl.runs),
-                       "replicas_per_run_per_gpu": R, "updates_per_step": U,
-                       "l2": "input X is 256 MiB, larger than L2; rows are gathered at random"},
+            "config": headline_config(wl, R, U),
             "roofline": roofline, "clocks": clocks,
             "gpu_launches": 2 * len(sims) * args.steps}
     for sim in sims:
