@@ -122,9 +122,11 @@ __global__ void __launch_bounds__(SWS_THREADS, 1) softmax_ws_kernel(NumericArgs 
   const int tiles_per_task = (m + T - 1) / T;
   bool failed = false;
 
+  if (warp >= NW) {
+  // the helper warpgroup gives registers up in one instruction that all four of its warps execute, then splits into roles
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(SWS_HELPER_REGS));
   if (warp == NW) {
     // =============================== producer warp: rows in ===============================
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(SWS_HELPER_REGS));
     ScheduleWalk walk;
     walk.done = true;
     int prod_st = 0;      // tiles are issued in order: the producer's stage is a counter
@@ -180,9 +182,8 @@ __global__ void __launch_bounds__(SWS_THREADS, 1) softmax_ws_kernel(NumericArgs 
       issue_tile();
       if (++st == S) { st = 0; par_empty ^= 1u; }
     }
-  } else if (warp > NW) {
+  } else {
     // =============================== softmax warps: two rows of the tile each ===============================
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(SWS_HELPER_REGS));
     __syncthreads();      // (1)
     __syncthreads();      // (2)
     const int sq = 2 * (warp - NW - 1) + (lane >> 4), sc = lane & 15;      // row of the tile, class; 16 lanes per row
@@ -236,6 +237,7 @@ __global__ void __launch_bounds__(SWS_THREADS, 1) softmax_ws_kernel(NumericArgs 
       if (++st == S) { st = 0; par_full ^= 1u; }
     }
     (void)par_full;
+  }
   } else {
     // =============================== FMA warps ===============================
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(SWS_FMA_REGS));
