@@ -531,7 +531,7 @@ sim_status sim_create(const sim_problem* problem, int32_t P, int32_t K, sim_vari
       if (prob.n_classes < 2 || prob.n_classes > SIM_MAX_CLASSES) return fail(nullptr, SIM_ERR_ARG, "n_classes must be in [2, SIM_MAX_CLASSES]");
     }
     if (prob.model == SIM_SOFTMAX) {
-      const char* why = softmax_shape_unsupported(prob.d, prob.n_classes, m);
+      const char* why = softmax_ws_supported(prob.d, prob.n_classes, m) ? nullptr : softmax_shape_unsupported(prob.d, prob.n_classes, m);
       if (why) return fail(nullptr, SIM_ERR_ARG, why);
     }
     if (prob.model == SIM_MLP2) {

@@ -66,6 +66,70 @@ __device__ __forceinline__ bool sws_wait(uint32_t bar, uint32_t parity, volatile
   return false;
 }
 
+// Parameters of a thread's pairs: global (row-major [C][d]) -> its own tensor-memory columns, zero where there is no such
+// pair / class.  Not inlined on purpose: in the asynchronous variants it is called inside the tile loop (a task with
+// another snapshot), and inlined there its loads in flight competed with the gradient accumulator for registers on every
+// tile; as a call the accumulator is saved and restored around it, where it is needed once per task.
+template <int KP>
+__device__ __noinline__ void sws_load_params(const float* src, int d, int C, int tid, uint32_t t_own) {
+  constexpr int NT = SWS_FMA_THREADS, CP = SMT_CP, WC = SMT_WC;
+  const int dp = d >> 1;
+#pragma unroll
+  for (int k = 0; k < KP; ++k) {
+    const int p = tid + NT * k;
+    float w[WC];
+#pragma unroll
+    for (int c = 0; c < CP; ++c) {
+      float2 v = make_float2(0.f, 0.f);
+      if (p < dp && c < C) v = reinterpret_cast<const float2*>(src + (size_t)c * d)[p];
+      w[2 * c] = v.x; w[2 * c + 1] = v.y;
+    }
+    tm_st20(t_own + k * WC, w);
+  }
+  tm_wait_st();
+}
+
+// Eq. 3 for the asynchronous variants: w_{j+1} = w_j - scale G goes from one version of the pool to another in global
+// memory (the snapshot in tensor memory is some worker's stale one, not w_j).  Gm holds the nine accumulated class slots of
+// the thread's pairs ([slot][pair]); the tenth is minus their sum.  Returns the thread's share of |w_{j+1} - w_ref|^2.
+// Not inlined, and fed through local memory, for the reason given at sws_load_params: once per update, never per tile.
+template <int KP>
+__device__ __noinline__ float sws_async_update(const uint64_t* Gm, const float* w_from, float* w_to, const float* w_ref, float scale,
+                                               int d, int C, int tid) {
+  constexpr int NT = SWS_FMA_THREADS, CP = SMT_CP, GC = CP - 1;
+  const int dp = d >> 1;
+  float dd = 0.f;
+#pragma unroll
+  for (int k = 0; k < KP; ++k) {
+    const int p = tid + NT * k;
+    if (p >= dp) continue;
+    float s0 = 0.f, s1 = 0.f;      // sum of the nine accumulated slots, in slot order
+#pragma unroll
+    for (int c = 0; c < CP; ++c) {
+      float g0, g1;
+      if (c < GC) {
+        unpack2(Gm[c * KP + k], g0, g1);
+        s0 += g0; s1 += g1;
+      } else {
+        g0 = C == CP ? -s0 : 0.f;
+        g1 = C == CP ? -s1 : 0.f;
+      }
+      if (c < C) {
+        float2 v = reinterpret_cast<const float2*>(w_from + (size_t)c * d)[p];
+        v.x = fmaf(-scale, g0, v.x);
+        v.y = fmaf(-scale, g1, v.y);
+        reinterpret_cast<float2*>(w_to + (size_t)c * d)[p] = v;
+        if (w_ref) {
+          const float2 wr = reinterpret_cast<const float2*>(w_ref + (size_t)c * d)[p];
+          const float e0 = v.x - wr.x, e1 = v.y - wr.y;
+          dd = fmaf(e0, e0, dd); dd = fmaf(e1, e1, dd);
+        }
+      }
+    }
+  }
+  return dd;
+}
+
 template <int KP, int TG, bool ASYNC>
 __global__ void __launch_bounds__(SWS_THREADS, 1) softmax_ws_kernel(NumericArgs a) {
   constexpr int NG = SWS_NG, NT = SWS_FMA_THREADS, NW = NT / 32, T = NG * TG, CP = SMT_CP, WC = SMT_WC, OWN = KP * WC, NV = TG * CP;
@@ -249,22 +313,7 @@ __global__ void __launch_bounds__(SWS_THREADS, 1) softmax_ws_kernel(NumericArgs 
     const uint32_t t_own = tmem + lane_base + (uint32_t)(grp * OWN);    // this thread's own columns
     const uint32_t t_lane = tmem + lane_base;                           // all columns of its lane
 
-    // parameters of this thread's pairs: global (row-major [C][d]) -> tensor memory, zero where there is no such pair / class
-    auto load_w = [&](const float* src) {
-#pragma unroll
-      for (int k = 0; k < KP; ++k) {
-        const int p = tid + NT * k;
-        float w[WC];
-#pragma unroll
-        for (int c = 0; c < CP; ++c) {
-          float2 v = make_float2(0.f, 0.f);
-          if (p < dp && c < C) v = reinterpret_cast<const float2*>(src + (size_t)c * d)[p];
-          w[2 * c] = v.x; w[2 * c + 1] = v.y;
-        }
-        tm_st20(t_own + k * WC, w);
-      }
-      tm_wait_st();
-    };
+    auto load_w = [&](const float* src) { sws_load_params<KP>(src, d, C, tid, t_own); };
     if (my_iters > 0) load_w(ASYNC ? a.pool + ((size_t)r * a.n_slots + *first_snap_s) * np : a.w_state + (size_t)r * np);
     tm_fence_before();
     __syncthreads();      // (2)
@@ -325,72 +374,79 @@ __global__ void __launch_bounds__(SWS_THREADS, 1) softmax_ws_kernel(NumericArgs 
       if (lane == 0) mbar_arrive(smem_addr(&empty[gst]));
     };
 
+    // logits of this group's rows (row grp + NG s of the tile, s < TG) over the features of its lane, for the tile in stage
+    // `lst`; the warp's partial sums go to buffer `lbuf` and are published
+    auto logit_pass = [&](int lst, int lbuf) {
+      const float* tile = rows_s + (size_t)lst * T * DS;
+      float acc[NV + 2];
+#pragma unroll
+      for (int i = 0; i < NV + 2; ++i) acc[i] = 0.f;
+      const float2* rowp = reinterpret_cast<const float2*>(tile + grp * DS) + L;
+#pragma unroll
+      for (int ck = 0; ck < NG * KP; ++ck) {
+        const int gp = ck / KP, k = ck % KP;
+        float w[WC];
+        tm_ld20(t_lane + ck * WC, w);
+        float2 x[TG];
+#pragma unroll
+        for (int s = 0; s < TG; ++s) x[s] = rowp[s * NG * (DS / 2) + 128 * gp + NT * k];
+        tm_wait_ld();
+#pragma unroll
+        for (int s = 0; s < TG; ++s) {
+#pragma unroll
+          for (int c = 0; c < CP; ++c)
+            acc[s * CP + c] = fmaf(x[s].y, w[2 * c + 1], fmaf(x[s].x, w[2 * c], acc[s * CP + c]));
+        }
+      }
+      tm_reduce_steps<16, NV>(acc, lane);
+      if (red_idx >= 0) red_s[(lbuf * NW + warp) * 32 + red_idx] = acc[0];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_addr(&zready[lbuf]));
+    };
+    // loss and distance of the update that ends with a tile of K contributors, recorded by thread 0 after the barrier
+    auto record = [&](int K_of_update) {
+      if (tid == 0) {
+        float tot = 0.f, ls = 0.f;
+        for (int w = 0; w < NW; ++w) tot += misc_s[w];
+        for (int q = 0; q < T; ++q) ls += lossrow_s[q];      // published with the update's last softmax terms
+        a.dist2[(size_t)r * a.cap + j] = a.w_ref ? tot : 0.f;
+        a.loss[(size_t)r * a.cap + j] = ls / ((float)K_of_update * (float)m);
+      }
+      ++j;
+    };
+
     int st = 0;
     uint32_t par_full = 0;
     bool pending = false;     // tile it - 1 still waits for its gradient pass
     int st_prev = 0;
-    for (long long it = 0; my_iters > 0; ++it) {
-      const int buf = (int)(it & 1);
-      if (!sws_wait(smem_addr(&full[st]), par_full, abort_s)) { failed = true; break; }
-      const TmTileInfo ti = info_s[st];
-      const float* tile = rows_s + (size_t)st * T * DS;
-
-      // ---- logits of this group's rows (row grp + NG s of the tile, s < TG) over the features of its lane ----
-      {
-        float acc[NV + 2];
-#pragma unroll
-        for (int i = 0; i < NV + 2; ++i) acc[i] = 0.f;
-        const float2* rowp = reinterpret_cast<const float2*>(tile + grp * DS) + L;
-#pragma unroll
-        for (int ck = 0; ck < NG * KP; ++ck) {
-          const int gp = ck / KP, k = ck % KP;
-          float w[WC];
-          tm_ld20(t_lane + ck * WC, w);
-          float2 x[TG];
-#pragma unroll
-          for (int s = 0; s < TG; ++s) x[s] = rowp[s * NG * (DS / 2) + 128 * gp + NT * k];
-          tm_wait_ld();
-#pragma unroll
-          for (int s = 0; s < TG; ++s) {
-#pragma unroll
-            for (int c = 0; c < CP; ++c)
-              acc[s * CP + c] = fmaf(x[s].y, w[2 * c + 1], fmaf(x[s].x, w[2 * c], acc[s * CP + c]));
-          }
+    if (!ASYNC) {
+      // ---- synchronous variants: one flat loop; the parameters change once per update, in tensor memory ----
+      for (long long it = 0; my_iters > 0; ++it) {
+        const int buf = (int)(it & 1);
+        if (!sws_wait(smem_addr(&full[st]), par_full, abort_s)) { failed = true; break; }
+        const TmTileInfo ti = info_s[st];
+        logit_pass(st, buf);
+        // gradient pass of the previous tile, whose softmax terms were formed while this one's logits ran
+        if (pending) {
+          if (!sws_wait(smem_addr(&dready[buf ^ 1]), (uint32_t)(((it - 1) >> 1) & 1), abort_s)) { failed = true; break; }
+          gradient_pass(st_prev, buf ^ 1);
         }
-        tm_reduce_steps<16, NV>(acc, lane);
-        if (red_idx >= 0) red_s[(buf * NW + warp) * 32 + red_idx] = acc[0];
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_addr(&zready[buf]));      // this warp's partial logits of tile it are published
-
-      // ---- gradient pass of the previous tile, whose softmax terms were formed while this one's logits ran ----
-      if (pending) {
-        if (!sws_wait(smem_addr(&dready[buf ^ 1]), (uint32_t)(((it - 1) >> 1) & 1), abort_s)) { failed = true; break; }
-        gradient_pass(st_prev, buf ^ 1);
-      }
-      pending = true;
-      st_prev = st;
-
-      const bool last_of_update = (ti.flags & TILE_LAST_OF_UPDATE) != 0;
-      const bool reload = ASYNC && (ti.flags & TILE_LAST_OF_TASK) && !(ti.flags & TILE_LAST_OF_RUN);
-      if (last_of_update || (ti.flags & TILE_LAST_OF_RUN)) {
-        // the update needs this tile's gradient too: the pipeline drains here
-        if (!sws_wait(smem_addr(&dready[buf]), (uint32_t)((it >> 1) & 1), abort_s)) { failed = true; break; }
-        gradient_pass(st, buf);
-        pending = false;
-      }
-      if (last_of_update || reload) {
-        if (!fma_barrier()) { failed = true; break; }     // every warp is through the logit pass that read these parameters
-        float dd = 0.f;
-        if (last_of_update) {
+        pending = true;
+        st_prev = st;
+        if (ti.flags & TILE_LAST_OF_UPDATE) {
+          // the update needs this tile's gradient too: the pipeline drains here
+          if (!sws_wait(smem_addr(&dready[buf]), (uint32_t)((it >> 1) & 1), abort_s)) { failed = true; break; }
+          gradient_pass(st, buf);
+          pending = false;
+          if (!fma_barrier()) { failed = true; break; }     // every warp is through the logit pass that read these parameters
           const float scale = (float)((double)a.eta / ((double)ti.K * (double)m));
-          const float* w_from = ASYNC ? a.pool + ((size_t)r * a.n_slots + cur_slot) * np : nullptr;
-          float* w_to = ASYNC ? a.pool + ((size_t)r * a.n_slots + ti.fresh) * np : nullptr;
+          float dd = 0.f;
 #pragma unroll
           for (int k = 0; k < KP; ++k) {
             const int p = tid + NT * k;
             float w[WC];
-            if (!ASYNC) { tm_ld20(t_own + k * WC, w); tm_wait_ld(); }
+            tm_ld20(t_own + k * WC, w);
+            tm_wait_ld();
             float s0 = 0.f, s1 = 0.f;      // sum of the nine accumulated slots, in slot order
 #pragma unroll
             for (int c = 0; c < CP; ++c) {
@@ -403,46 +459,80 @@ __global__ void __launch_bounds__(SWS_THREADS, 1) softmax_ws_kernel(NumericArgs 
                 g0 = C == CP ? -s0 : 0.f;
                 g1 = C == CP ? -s1 : 0.f;
               }
-              if (ASYNC) {
-                if (p < dp && c < C) {
-                  float2 v = reinterpret_cast<const float2*>(w_from + (size_t)c * d)[p];
-                  v.x = fmaf(-scale, g0, v.x);
-                  v.y = fmaf(-scale, g1, v.y);
-                  reinterpret_cast<float2*>(w_to + (size_t)c * d)[p] = v;
-                  w[2 * c] = v.x; w[2 * c + 1] = v.y;
-                }
-              } else {
-                w[2 * c] = fmaf(-scale, g0, w[2 * c]);
-                w[2 * c + 1] = fmaf(-scale, g1, w[2 * c + 1]);
-              }
+              w[2 * c] = fmaf(-scale, g0, w[2 * c]);
+              w[2 * c + 1] = fmaf(-scale, g1, w[2 * c + 1]);
               if (a.w_ref && p < dp && c < C) {
                 const float2 wr = reinterpret_cast<const float2*>(a.w_ref + (size_t)c * d)[p];
                 const float e0 = w[2 * c] - wr.x, e1 = w[2 * c + 1] - wr.y;
                 dd = fmaf(e0, e0, dd); dd = fmaf(e1, e1, dd);
               }
             }
-            if (!ASYNC) tm_st20(t_own + k * WC, w);
+            tm_st20(t_own + k * WC, w);
           }
-          if (ASYNC) cur_slot = ti.fresh;
+          dd = warp_sum(dd);
+          if (lane == 0) misc_s[warp] = dd;
+          tm_wait_st();
+          if (!fma_barrier()) { failed = true; break; }     // the parameters in tensor memory are the next tile's
+          record(ti.K);
+        }
+        if (ti.flags & TILE_LAST_OF_RUN) break;
+        if (++st == S) { st = 0; par_full ^= 1u; }
+      }
+    } else {
+      // ---- asynchronous variants: every task brings another snapshot, so the parameters change every few tiles.  The
+      //      tile loop is kept free of the reload's and the update's calls and global traffic: with them inside it, the
+      //      loop's own state lived on the stack (17 local loads and stores a tile, 40 % more time per row) ----
+      long long it = 0;
+      bool running = my_iters > 0;
+      while (running) {
+        TmTileInfo ti;
+        int buf;
+        for (;;) {
+          buf = (int)(it & 1);
+          if (!sws_wait(smem_addr(&full[st]), par_full, abort_s)) { failed = true; break; }
+          ti = info_s[st];
+          logit_pass(st, buf);
+          if (pending) {
+            if (!sws_wait(smem_addr(&dready[buf ^ 1]), (uint32_t)(((it - 1) >> 1) & 1), abort_s)) { failed = true; break; }
+            gradient_pass(st_prev, buf ^ 1);
+          }
+          pending = true;
+          st_prev = st;
+          if (ti.flags & TILE_LAST_OF_TASK) break;          // (the last tile of an update or of the run is the last of a task)
+          ++it;
+          if (++st == S) { st = 0; par_full ^= 1u; }
+        }
+        if (failed) break;
+        const bool last_of_update = (ti.flags & TILE_LAST_OF_UPDATE) != 0;
+        const bool reload = !(ti.flags & TILE_LAST_OF_RUN);
+        if (last_of_update) {
+          if (!sws_wait(smem_addr(&dready[buf]), (uint32_t)((it >> 1) & 1), abort_s)) { failed = true; break; }
+          gradient_pass(st, buf);
+          pending = false;
+        }
+        if (!fma_barrier()) { failed = true; break; }       // every warp is through the logit pass that read these parameters
+        if (last_of_update) {
+          // the accumulator goes through local memory into a call (see sws_async_update) and starts again at zero
+          const float scale = (float)((double)a.eta / ((double)ti.K * (double)m));
+          uint64_t Gm[GC * KP];
+#pragma unroll
+          for (int c = 0; c < GC; ++c)
+#pragma unroll
+            for (int k = 0; k < KP; ++k) { Gm[c * KP + k] = G[c][k]; G[c][k] = 0ull; }
+          float dd = sws_async_update<KP>(Gm, a.pool + ((size_t)r * a.n_slots + cur_slot) * np,
+                                          a.pool + ((size_t)r * a.n_slots + ti.fresh) * np, a.w_ref, scale, d, C, tid);
+          cur_slot = ti.fresh;
           dd = warp_sum(dd);
           if (lane == 0) misc_s[warp] = dd;
         }
         if (reload) load_w(a.pool + ((size_t)r * a.n_slots + ti.next_snap) * np);   // the next task's snapshot (own elements only)
         tm_wait_st();
-        if (!fma_barrier()) { failed = true; break; }     // the parameters in tensor memory are the next tile's
-        if (last_of_update) {
-          if (tid == 0) {
-            float tot = 0.f, ls = 0.f;
-            for (int w = 0; w < NW; ++w) tot += misc_s[w];
-            for (int q = 0; q < T; ++q) ls += lossrow_s[q];      // published with this tile's softmax terms
-            a.dist2[(size_t)r * a.cap + j] = a.w_ref ? tot : 0.f;
-            a.loss[(size_t)r * a.cap + j] = ls / ((float)ti.K * (float)m);
-          }
-          ++j;
-        }
+        if (!fma_barrier()) { failed = true; break; }       // the parameters in tensor memory are the next tile's
+        if (last_of_update) record(ti.K);
+        if (ti.flags & TILE_LAST_OF_RUN) running = false;
+        ++it;
+        if (++st == S) { st = 0; par_full ^= 1u; }
       }
-      if (ti.flags & TILE_LAST_OF_RUN) break;
-      if (++st == S) { st = 0; par_full ^= 1u; }
     }
 
     if (!failed && !ASYNC && my_iters > 0) {
