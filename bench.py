@@ -377,8 +377,13 @@ def run_profile_case(args, wl):
     data = wl.make_data()
     dev = device_data(data)
     variant, K = wl.runs[args.profile_run]
+    if args.profile_variant:
+        variant, K = args.profile_variant, args.profile_K
     R = args.profile_replicas or wl.replicas
-    sim = make_sim(wl, dev, variant, K, R, interval=args.profile_interval or None)
+    interval = args.profile_interval or None
+    if args.profile_variant and wl.t_interval > 0:
+        interval = 0.0                   # a given (variant, K) is run as it is, without the AdaSync rule
+    sim = make_sim(wl, dev, variant, K, R, interval=interval)
     J = args.profile_updates
     sim.reserve(J)
     torch.cuda.synchronize()
@@ -415,6 +420,9 @@ def main():
                          "--profile-updates updates (a capture-sized case for ncu) and print its device time")
     ap.add_argument("--profile-n", type=int, default=65536, help="samples of the profile case (0: the workload's)")
     ap.add_argument("--profile-run", type=int, default=0, help="which of the workload's (variant, K) runs")
+    ap.add_argument("--profile-variant", default="", choices=["", "ksync", "kbatchsync", "kasync", "kbatchasync"],
+                    help="run the profile case with this variant and --profile-K instead of one of the workload's runs")
+    ap.add_argument("--profile-K", type=int, default=4)
     ap.add_argument("--profile-updates", type=int, default=3)
     ap.add_argument("--profile-replicas", type=int, default=0)
     ap.add_argument("--profile-interval", type=float, default=0.0, help="AdaSync interval of the profile case (default: the workload's)")
