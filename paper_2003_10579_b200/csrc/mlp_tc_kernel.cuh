@@ -1,23 +1,5 @@
-// MLP forward pass on the 5th-generation tensor cores (tcgen05) with the accumulator in tensor
-// memory.
-//
-// One CTA per (replica, contributor, 128-sample block):  A1[128 x H] = bf16(X_b)[128 x d] bf16(W1)[d x H]
-//   warp 0   B producer: TMA tensor loads of W1 from the transposed, k-block-tiled bf16 shadow (K-major B
-//            operand, 128-byte swizzle), half a k-block ([H/2 x 64], contiguous in the shadow) per ring
-//            slot; the first slots are requested before the block's opening barrier
-//   warps 2-5  A producer during the main loop: the 128 gathered sample rows of a k-block are 1024
-//            16-byte pieces, copied with cp.async into the same 128-byte-swizzle pattern (one-row
-//            TMA boxes of 128 B were limited by the TMA instruction rate), made visible to the
-//            tensor core's asynchronous proxy with a proxy fence before the slot is signalled
-//   warp 1   allocates tensor memory; one elected lane issues tcgen05.mma (M=128, N<=256, K=16)
-//            and commits slot-free / accumulator-ready mbarriers
-//   warps 6-9  during the main loop: stage b1, W2 (padded to 16 classes) and b2 of the snapshot
-//   warps 2-9  epilogue: tcgen05.ld gives each thread one sample's row of A1 - warps 2-5 the first
-//            half of the hidden units, warps 6-9 the second - so bias, relu and the partial logits
-//            need no cross-thread reduction; the two partial logit vectors of a row meet in shared
-//            memory, both threads form softmax and delta2, and a second pass over tensor memory
-//            forms delta1 = (delta2 W2^T) . [A1 + b1 > 0] for the own half, stores it in bf16 and
-//            reduces its column sums (db1) with a warp transposition reduce
+// The MLP's two products over d on the 5th-generation tensor cores (tcgen05), accumulators in tensor memory:
+// mlp_forward_tc_kernel (training, persistent), mlp_risk_tc_kernel (forward-only, full-data risk), mlp_dw1_tc_kernel.
 // Every mbarrier wait is bounded; a wait that runs out sets the error word and the CTA drains.
 #pragma once
 #include <cuda.h>
@@ -108,33 +90,31 @@ inline __host__ __device__ TcLayout tc_forward_layout(int H) {
 }
 static_assert(512 * 16 * 4 + 2 * 128 * 16 * 4 <= 4 * TC_A_BYTES, "W2 and the partial logits must fit the A ring's bytes");
 
-// EVAL = true is the forward-only form for the full-data risk F(w) of Eq. 1: one CTA per (replica, 128 consecutive rows
-// of the data set), the replica's current version, and only the rows' losses leave the CTA.
-template <bool EVAL>
+// Forward-only pass for the full-data risk F(w) of Eq. 1: one CTA per (replica, 128 consecutive rows of the data set),
+// A1[128 x H] = bf16(X_b)[128 x d] bf16(W1)[d x H] with the replica's current version; only the rows' losses leave the CTA.
+//   warp 0   B producer: TMA tensor loads of W1 from the transposed, k-block-tiled bf16 shadow (K-major B
+//            operand, 128-byte swizzle), half a k-block ([H/2 x 64], contiguous in the shadow) per ring
+//            slot; the first slots are requested before the block's opening barrier
+//   warps 2-5  A producer during the main loop: the 128 sample rows of a k-block are 1024
+//            16-byte pieces, copied with cp.async into the same 128-byte-swizzle pattern, made visible to the
+//            tensor core's asynchronous proxy with a proxy fence before the slot is signalled
+//   warp 1   allocates tensor memory; one elected lane issues tcgen05.mma (M=128, N<=256, K=16)
+//            and commits slot-free / accumulator-ready mbarriers
+//   warps 6-9  during the main loop: stage b1, W2 (padded to 16 classes) and b2
+//   warps 2-9  epilogue: tcgen05.ld gives each thread one sample's row of A1 - warps 2-5 the first
+//            half of the hidden units, warps 6-9 the second - so bias, relu and the partial logits
+//            need no cross-thread reduction; the two partial logit vectors of a row meet in shared
+//            memory and the row's softmax cross-entropy is summed per warp
 __global__ void __launch_bounds__(TC_THREADS, 1)
-mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmW, MlpArgs g) {
+mlp_risk_tc_kernel(const __grid_constant__ CUtensorMap tmW, MlpArgs g) {
   const NumericArgs& a = g.na;
   const MlpScratch& sc = g.sc;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int H = sc.H, C = sc.C, d = sc.d, m = sc.m;
-  const int mtiles = EVAL ? g.eval_blocks : m / 128;
+  const int H = sc.H, C = sc.C, d = sc.d;
+  const int mtiles = g.eval_blocks;
   const int mt = blockIdx.x % mtiles;
-  const int l = EVAL ? 0 : (blockIdx.x / mtiles) % sc.Kmax;
-  const int r = EVAL ? blockIdx.x / mtiles : blockIdx.x / (mtiles * sc.Kmax);
-  const long long j = g.j;
-  uint32_t worker = 0, seq = 0;
-  int snap;
-  if (EVAL) {
-    snap = g.eval_slot ? (int)g.eval_slot[r] : g.eval_parity;
-  } else {
-    const int K = (int)a.K_used[(size_t)r * a.cap + j];
-    if (l >= K) return;
-    const size_t ent = ((size_t)r * a.cap + j) * a.K_stride + l;
-    worker = a.worker[ent]; seq = a.seq[ent];
-    snap = mlp_snap_slot(a, r, j, l);
-  }
-  const uint32_t rid = a.replica_base + (uint32_t)r;
-  const size_t task = (size_t)r * sc.Kmax + l;
+  const int r = blockIdx.x / mtiles;
+  const int snap = g.eval_slot ? (int)g.eval_slot[r] : g.eval_parity;
   const long long dH = (long long)d * H;
   const float* wsnap = a.pool + ((size_t)r * a.n_slots + snap) * a.slot_stride;
   const int n_halves = H > 256 ? 2 : 1;
@@ -179,16 +159,11 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmW, MlpArgs g) {
     }
   }
   if (warp == 1) tc_alloc(smem_addr(tmem_slot), tmem_cols);
-  if (tid >= 64 && tid < 192) {                     // the minibatch: sample rows and labels (the A producers need them first)
+  if (tid >= 64 && tid < 192) {                     // sample rows and labels (the A producers need them first)
     const int t = tid - 64;
-    uint32_t idx;
-    if (EVAL) {     // consecutive rows; a row past the end of the data set repeats the last one and is left out of the sum
-      const uint64_t want = (uint64_t)mt * 128 + t;
-      idx = (uint32_t)(want < a.n ? want : a.n - 1);
-    } else {
-      idx = draw_index(a.seed, rid, worker, seq, (uint32_t)(mt * 128 + t), a.n);
-      if ((uint64_t)idx >= a.n) { atomicExch(a.err, ERR_BAD_INDEX); idx = 0; }
-    }
+    // consecutive rows; a row past the end of the data set repeats the last one and is left out of the sum
+    const uint64_t want = (uint64_t)mt * 128 + t;
+    const uint32_t idx = (uint32_t)(want < a.n ? want : a.n - 1);
     rows_s[t] = (int)idx;
     label_s[t] = reinterpret_cast<const int*>(a.y)[idx];
   }
@@ -240,8 +215,6 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmW, MlpArgs g) {
     const int q = warp & 3;                         // the TMEM lane quarter this warp may read
     const int ehalf = warp >= 6 ? 1 : 0;            // hidden units [ehalf * H/2, +H/2)
     const int row = 32 * q + lane;
-    const size_t grow = task * m + (size_t)mt * 128 + row;
-    const int part = mt * 4 + q, parts = mtiles * 4;
     if (ehalf) {
       // ---- helpers: b1 and b2 of the snapshot during the main loop; W2 (rows padded to 16 classes) goes into the A
       //      ring's bytes once the last MMA has read them (its values wait in registers meanwhile) ----
@@ -304,7 +277,6 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmW, MlpArgs g) {
       for (int c = 0; c < 16; ++c) z[c] = 0.f;
       for (int ch = ch0; ch < ch1; ++ch) {
         tc_ld32(trow + ch * 32, v);
-        float4* hout = reinterpret_cast<float4*>(sc.Hact + grow * H + ch * 32);
 #pragma unroll
         for (int i4 = 0; i4 < 8; ++i4) {
           float hv[4];
@@ -322,7 +294,6 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmW, MlpArgs g) {
               }
             }
           }
-          if (!EVAL) hout[i4] = make_float4(hv[0], hv[1], hv[2], hv[3]);
         }
       }
 #pragma unroll
@@ -331,84 +302,15 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmW, MlpArgs g) {
     }
     group_barrier(1, 256);                          // both halves of every row's logits are published
     if (!failed) {
-      // logits = b2 + half 0 + half 1, in this order in both threads of the row
+      // logits = b2 + half 0 + half 1
 #pragma unroll
       for (int c = 0; c < 16; ++c) z[c] = (b2_s[c] + zx_s[row * 16 + c]) + zx_s[(128 + row) * 16 + c];
-      // softmax cross-entropy of this row; exponentials without the maximal class keep log(1+s)
-      // and p_max - 1 = -s/(1+s) accurate for wide margins
-      const int lab = label_s[row];
-      float zmax = -INFINITY;
-#pragma unroll
-      for (int c = 0; c < 16; ++c) { if (c >= C) z[c] = -INFINITY; zmax = fmaxf(zmax, z[c]); }
-      int cmax = 0;
-#pragma unroll
-      for (int c = 15; c >= 0; --c) if (c < C && z[c] == zmax) cmax = c;
-      float zl = 0.f;
-#pragma unroll
-      for (int c = 0; c < 16; ++c) if (c == lab) zl = z[c];
-      float sexcl = 0.f;
-#pragma unroll
-      for (int c = 0; c < 16; ++c) { z[c] = (c < C && c != cmax) ? expf(z[c] - zmax) : 0.f; sexcl += z[c]; }
-      if (EVAL) {     // the row's loss is all that is wanted
-        if (!ehalf) {
-          const bool real = (uint64_t)mt * 128 + row < a.n;
-          const float rowloss = warp_sum(real ? log1pf(sexcl) + (zmax - zl) : 0.f);
-          if (lane == 0) g.eval_part[((size_t)r * g.eval_blocks + mt) * 4 + q] = rowloss;
-        }
-      } else {
-      const float ssum = 1.f + sexcl;
-      float d2[16];
-#pragma unroll
-      for (int c = 0; c < 16; ++c) {
-        float dl = 0.f;
-        if (c < C) {
-          if (c == cmax) dl = c == lab ? -sexcl / ssum : 1.f / ssum;
-          else dl = z[c] / ssum - (c == lab ? 1.f : 0.f);
-        }
-        d2[c] = dl;
-      }
       if (!ehalf) {
-#pragma unroll
-        for (int c4 = 0; c4 < 4; ++c4)
-          reinterpret_cast<float4*>(sc.D2 + grow * 16)[c4] = make_float4(d2[4 * c4], d2[4 * c4 + 1], d2[4 * c4 + 2], d2[4 * c4 + 3]);
-        float rowloss = warp_sum(log1pf(sexcl) + (zmax - zl));
-        if (lane == 0) sc.loss_part[task * parts + part] = rowloss;
-      }
-
-      // second pass: delta1, its bf16 copy and its column sums over this warp's 32 rows, own half of the units
-      for (int ch = ch0; ch < ch1; ++ch) {
-        tc_ld32(trow + ch * 32, v);
-        float dv[32];
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const int col = ch * 32 + i;
-          const float a1 = __uint_as_float(v[i]) + b1_s[col];
-          const float4* wr = reinterpret_cast<const float4*>(W2_s + col * 16);
-          float acc = 0.f;
-#pragma unroll
-          for (int c4 = 0; c4 < 4; ++c4) {
-            if (4 * c4 < C) {
-              const float4 w = wr[c4];
-              acc = fmaf(d2[4 * c4], w.x, acc); acc = fmaf(d2[4 * c4 + 1], w.y, acc);
-              acc = fmaf(d2[4 * c4 + 2], w.z, acc); acc = fmaf(d2[4 * c4 + 3], w.w, acc);
-            }
-          }
-          dv[i] = a1 > 0.f ? acc : 0.f;
-        }
-        uint4* dout = reinterpret_cast<uint4*>(sc.D1q + grow * H + ch * 32);
-#pragma unroll
-        for (int i8 = 0; i8 < 4; ++i8) {
-          uint32_t pk[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const __nv_bfloat162 b = __floats2bfloat162_rn(dv[i8 * 8 + 2 * e], dv[i8 * 8 + 2 * e + 1]);
-            pk[e] = *reinterpret_cast<const uint32_t*>(&b);
-          }
-          dout[i8] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-        }
-        warp_transpose_reduce(dv, lane);
-        sc.db1_part[(task * parts + part) * H + ch * 32 + lane] = dv[0];
-      }
+        float d2[16];
+        const bool real = (uint64_t)mt * 128 + row < a.n;
+        const float loss = mlp_row_softmax<false>(z, C, label_s[row], d2);
+        const float rowloss = warp_sum(real ? loss : 0.f);
+        if (lane == 0) g.eval_part[((size_t)r * g.eval_blocks + mt) * 4 + q] = rowloss;
       }
     }
   }
@@ -419,6 +321,259 @@ mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmW, MlpArgs g) {
   if (failed && lane == 0) atomicExch(a.err, ERR_WAIT_TIMEOUT);
 }
 
+
+
+// Position in a ring of n slots: slot and phase parity of use number u, stepped as counters (u % n and u / n with a
+// run-time n and a 64-bit u are a division subroutine each, on the critical path of single-thread roles).
+struct RingPos {
+  int s;
+  uint32_t ph;
+  __device__ __forceinline__ void step(int n, int by = 1) { s += by; if (s >= n) { s -= n; ph ^= 1u; } }
+};
+
+
+// ---- training forward pass: persistent kernel --------------------------------------------------------------------
+// Tiles of one (replica, contributor, 128-sample block) x Hn hidden units (Hn = H, or H/2 for H > 256) are dealt round-robin
+// to one CTA per SM; the two halves of a block are neighbours in that order, so that the second reader of the block's
+// sample rows finds them in L2.  The accumulator is double-buffered in tensor memory: the epilogue of one tile runs under
+// the loads and MMAs of the next.  The epilogue gives each thread one sample's row of A1 (tcgen05.ld 32x32b), so bias, relu
+// and the tile's share of the logits h W2 need no cross-thread reduction; h and the partial logits go to global memory and
+// the head kernel takes it from there (softmax needs all hidden units of a row, which no single tile has).
+//   warp 0      TMA producer of B: [Hn x 64] blocks of the transposed, k-block-tiled bf16 shadow of W1 (K-major operand,
+//               128-byte swizzle), one ring slot per k-block
+//   warp 1      allocates tensor memory; one elected lane issues tcgen05.mma (M = 128, N = Hn, K = 16) and commits the
+//               slot-free / accumulator-ready mbarriers
+//   warps 2-5   A producers: the 128 gathered sample rows of a k-block are 1024 16-byte pieces, copied with cp.async into
+//               the 128-byte-swizzle pattern (one-row TMA boxes of 128 B were limited by the TMA instruction rate) and
+//               made visible to the tensor core's asynchronous proxy with a proxy fence before the slot is signalled
+//   warps 6-9   epilogue (one warp per tensor-memory lane quarter): stage b1 and W2 (rows padded to 16 classes) of the
+//               tile's snapshot and hidden units in shared memory, wait for the accumulator, form h and the partial logits
+struct TcFwdLayout { int sa, sb, b_bytes, off_b, off_w2, off_b1, off_bars, off_tmem, off_fail, total; };
+inline __host__ __device__ TcFwdLayout tc_fwd_layout(int H) {
+  TcFwdLayout L;
+  const int Hn = H > 256 ? H / 2 : H;
+  const int budget = 226 << 10;
+  L.b_bytes = Hn * 128;
+  L.sa = 4;
+  const int fixed = L.sa * TC_A_BYTES + Hn * 64 + Hn * 4 + 8 * (2 * L.sa + 2 * 8 + 4) + 32 + 1024;
+  L.sb = (budget - fixed) / L.b_bytes;
+  if (L.sb > 8) L.sb = 8;
+  L.off_b = L.sa * TC_A_BYTES;
+  L.off_w2 = L.off_b + L.sb * L.b_bytes;          // [Hn][16] floats
+  L.off_b1 = L.off_w2 + Hn * 64;
+  L.off_bars = L.off_b1 + Hn * 4;
+  L.off_tmem = L.off_bars + 8 * (2 * L.sa + 2 * L.sb + 4);
+  L.off_fail = L.off_tmem + 16;
+  L.total = L.off_fail + 16 + 1024;               // slack for the manual 1024-byte alignment
+  return L;
+}
+
+__global__ void __launch_bounds__(TC_THREADS, 1)
+mlp_forward_tc_kernel(const __grid_constant__ CUtensorMap tmW, MlpArgs g) {
+  const NumericArgs& a = g.na;
+  const MlpScratch& sc = g.sc;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int H = sc.H, C = sc.C, d = sc.d, m = sc.m;
+  const int mtiles = m / 128, n_halves = H > 256 ? 2 : 1, Hn = H / n_halves;
+  const int n_tiles = a.R * sc.Kmax * mtiles * n_halves;
+  const int nk = d / TC_BK;
+  const long long j = g.j;
+  const long long dH = (long long)d * H;
+  uint32_t tmem_cols = 32;
+  while ((int)tmem_cols < 2 * Hn) tmem_cols <<= 1;
+
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw_addr = smem_addr(smem_raw);
+  const uint32_t base_addr = (raw_addr + 1023u) & ~1023u;
+  unsigned char* base = smem_raw + (base_addr - raw_addr);
+  const TcFwdLayout L = tc_fwd_layout(H);
+  const int SA = L.sa, SB = L.sb;
+  float* W2_s = reinterpret_cast<float*>(base + L.off_w2);
+  float* b1_s = reinterpret_cast<float*>(base + L.off_b1);
+  const uint32_t bars = base_addr + L.off_bars;      // afull[SA] | aempty[SA] | bfull[SB] | bempty[SB] | acc_full[2] | acc_empty[2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base + L.off_tmem);
+  volatile int* fail_s = reinterpret_cast<volatile int*>(base + L.off_fail);
+  auto afull = [&](int s) { return bars + 8u * s; };
+  auto aempty = [&](int s) { return bars + 8u * (SA + s); };
+  auto bfull = [&](int s) { return bars + 8u * (2 * SA + s); };
+  auto bempty = [&](int s) { return bars + 8u * (2 * SA + SB + s); };
+  auto acc_full = [&](int b) { return bars + 8u * (2 * SA + 2 * SB + b); };
+  auto acc_empty = [&](int b) { return bars + 8u * (2 * SA + 2 * SB + 2 + b); };
+
+  if (tid == 0) {
+    // an A slot is full after its 128 producer threads arrived, a B slot after the TMA bytes (one arrival with expect_tx)
+    for (int s = 0; s < SA; ++s) { mbar_init(afull(s), 128); mbar_init(aempty(s), 1); }
+    for (int s = 0; s < SB; ++s) { mbar_init(bfull(s), 1); mbar_init(bempty(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 4); }
+    fail_s[0] = 0;
+    mbar_fence_init();
+  }
+  if (warp == 1) tc_alloc(smem_addr(tmem_slot), tmem_cols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  bool failed = false;
+  // tile t -> (replica r, contributor l, sample block mt, half hf of the hidden units); false for a contributor the
+  // update does not have (l >= K), which every role skips alike
+  auto tile_of = [&](int t, int& r, int& l, int& mt, int& hf) {
+    hf = t % n_halves;
+    int x = t / n_halves;
+    mt = x % mtiles; x /= mtiles;
+    l = x % sc.Kmax;
+    r = x / sc.Kmax;
+    return l < (int)a.K_used[(size_t)r * a.cap + j];
+  };
+
+  if (warp == 0) {
+    // ---- B producer ----
+    if (lane == 0) {
+      RingPos rp{0, 0u};
+      for (int t = blockIdx.x; t < n_tiles && !failed; t += gridDim.x) {
+        int r, l, mt, hf;
+        if (!tile_of(t, r, l, mt, hf)) continue;
+        const long long w_blk0 = ((long long)r * sc.n_slots + mlp_snap_slot(a, r, j, l)) * nk;     // first k-block of this W1^T shadow
+        for (int kc = 0; kc < nk; ++kc, rp.step(SB)) {
+          const int s = rp.s;
+          if (!mbar_wait(bempty(s), rp.ph ^ 1u)) { failed = true; break; }
+          mbar_arrive_expect_tx(bfull(s), (uint32_t)L.b_bytes);
+          tma_load_2d(base_addr + L.off_b + (uint32_t)s * L.b_bytes, &tmW, 0, (int)((w_blk0 + kc) * H + hf * Hn), bfull(s));
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ---- MMA issuer ----
+    const uint32_t idesc = tc_idesc(Hn, 0, 0);
+    RingPos ra{0, 0u}, rb{0, 0u};
+    int i = 0;
+    for (int t = blockIdx.x; t < n_tiles && !failed; t += gridDim.x) {
+      int r, l, mt, hf;
+      if (!tile_of(t, r, l, mt, hf)) continue;
+      const int buf = i & 1;
+      if (!mbar_wait(acc_empty(buf), (uint32_t)(((i >> 1) & 1) ^ 1))) { failed = true; break; }
+      tc_fence_after();
+      for (int kc = 0; kc < nk; ++kc, ra.step(SA), rb.step(SB)) {
+        if (!mbar_wait(afull(ra.s), ra.ph) || !mbar_wait(bfull(rb.s), rb.ph)) { failed = true; break; }
+        tc_fence_after();
+        if (lane == 0) {
+          const uint32_t As = base_addr + (uint32_t)ra.s * TC_A_BYTES, Bs = base_addr + L.off_b + (uint32_t)rb.s * L.b_bytes;
+#pragma unroll
+          for (int k16 = 0; k16 < TC_BK / 16; ++k16)
+            tc_mma_bf16(tmem_base + (uint32_t)(buf * Hn), tc_desc_kmajor(As + k16 * 32), tc_desc_kmajor(Bs + k16 * 32), idesc,
+                        (kc > 0 || k16 > 0) ? 1u : 0u);
+          tc_commit(bempty(rb.s));                  // the slots may be refilled once these MMAs have read them
+          tc_commit(aempty(ra.s));
+          if (kc == nk - 1) tc_commit(acc_full(buf));
+        }
+        __syncwarp();
+      }
+      ++i;
+    }
+  } else if (warp < 6) {
+    // ---- A producers: thread p copies 16-byte piece (p & 7) of rows (p >> 3) + 16 i, i < 8.  A k-block is
+    //      signalled FWD_LAG k-blocks after it was issued; the ring is deeper than that (SA > FWD_LAG + 1), so
+    //      the signal never waits for a slot whose release depends on the k-block just before the signalled one.
+    const int p = tid - 64, piece = p & 7, row0 = p >> 3;
+    long long it = 0, signalled = 0;
+    RingPos rp{0, 0u}, sig{0, 0u};
+    auto signal = [&]() {                 // the oldest unsignalled k-block has landed: publish to the async proxy
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      mbar_arrive(afull(sig.s));
+      sig.step(SA);
+      ++signalled;
+    };
+    for (int t = blockIdx.x; t < n_tiles && !failed; t += gridDim.x) {
+      int r, l, mt, hf;
+      if (!tile_of(t, r, l, mt, hf)) continue;
+      const int* rows = sc.rows_tab + ((size_t)r * sc.Kmax + l) * m + (size_t)mt * 128;
+      const __nv_bfloat16* src[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) src[i] = sc.Xq + (size_t)rows[row0 + 16 * i] * d + piece * 8;
+      for (int kc = 0; kc < nk; ++kc, ++it, rp.step(SA)) {
+        if (!mbar_wait(aempty(rp.s), rp.ph ^ 1u)) { failed = true; break; }
+        const uint32_t As = base_addr + (uint32_t)rp.s * TC_A_BYTES;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int rw = row0 + 16 * i;
+          cp_async16(As + rw * 128 + ((piece ^ (rw & 7)) << 4), src[i] + (size_t)kc * TC_BK);
+        }
+        cp_async_commit();
+        if (it >= FWD_LAG) {
+          cp_async_wait<FWD_LAG>();
+          signal();
+        }
+      }
+    }
+    cp_async_wait<0>();
+    if (!failed) while (signalled < it) signal();
+  } else {
+    // ---- epilogue: thread = one sample row of the tile ----
+    const int q = warp & 3;                         // the tensor-memory lane quarter this warp may read
+    const int row = 32 * q + lane, e0 = tid - 192;
+    for (int e = e0; e < Hn * 16; e += 128) W2_s[e] = 0.f;      // the padding classes stay zero
+    group_barrier(1, 128);
+    int i = 0;
+    for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+      int r, l, mt, hf;
+      if (!tile_of(t, r, l, mt, hf)) continue;
+      const int buf = i & 1;
+      const float* b1 = a.pool + ((size_t)r * a.n_slots + mlp_snap_slot(a, r, j, l)) * a.slot_stride + dH + hf * Hn;
+      const float* W2 = b1 + (H - hf * Hn) + (size_t)hf * Hn * C;
+      for (int e = e0; e < Hn; e += 128) b1_s[e] = b1[e];
+      for (int e = e0; e < Hn * C; e += 128) {
+        const int col = e / C;
+        W2_s[col * 16 + (e - col * C)] = W2[e];
+      }
+      if (!mbar_wait(acc_full(buf), (uint32_t)((i >> 1) & 1))) fail_s[0] = 1;
+      group_barrier(1, 128);                        // b1 / W2 are staged; the four warps give up together or not at all
+      if (fail_s[0]) { failed = true; break; }
+      tc_fence_after();
+      const size_t grow = ((size_t)r * sc.Kmax + l) * m + (size_t)mt * 128 + row;
+      const uint32_t trow = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * Hn);
+      float z[16];
+#pragma unroll
+      for (int c = 0; c < 16; ++c) z[c] = 0.f;
+      for (int ch = 0; ch < Hn / 32; ++ch) {
+        uint32_t v[32];
+        tc_ld32(trow + ch * 32, v);
+        float4* hout = reinterpret_cast<float4*>(sc.Hact + grow * H + hf * Hn + ch * 32);
+#pragma unroll
+        for (int i4 = 0; i4 < 8; ++i4) {
+          float hv[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int col = ch * 32 + i4 * 4 + e;
+            hv[e] = fmaxf(__uint_as_float(v[i4 * 4 + e]) + b1_s[col], 0.f);
+            const float4* wr = reinterpret_cast<const float4*>(W2_s + col * 16);
+#pragma unroll
+            for (int c4 = 0; c4 < 4; ++c4) {
+              if (4 * c4 < C) {
+                const float4 w = wr[c4];
+                z[4 * c4] = fmaf(hv[e], w.x, z[4 * c4]); z[4 * c4 + 1] = fmaf(hv[e], w.y, z[4 * c4 + 1]);
+                z[4 * c4 + 2] = fmaf(hv[e], w.z, z[4 * c4 + 2]); z[4 * c4 + 3] = fmaf(hv[e], w.w, z[4 * c4 + 3]);
+              }
+            }
+          }
+          hout[i4] = make_float4(hv[0], hv[1], hv[2], hv[3]);
+        }
+      }
+      tc_fence_before();                            // this warp's reads of the buffer are done: hand it back
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty(buf));
+#pragma unroll
+      for (int c4 = 0; c4 < 4; ++c4)
+        reinterpret_cast<float4*>(sc.ZP + (grow * n_halves + hf) * 16)[c4] = make_float4(z[4 * c4], z[4 * c4 + 1], z[4 * c4 + 2], z[4 * c4 + 3]);
+      group_barrier(1, 128);                        // b1 / W2 may be overwritten for the next tile
+      ++i;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tc_dealloc(tmem_base, tmem_cols);
+  if (failed && lane == 0) atomicExch(a.err, ERR_WAIT_TIMEOUT);
+}
 
 // Shared-memory matrix descriptor, 128-byte swizzle, MN-major operand (the M or N index is the
 // contiguous one): 64-element (128-byte) runs along MN, 8 such k-rows form a 1024-byte atom;
@@ -478,14 +633,6 @@ __device__ __forceinline__ void bulk_s2g(void* dst, uint32_t src, uint32_t bytes
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-// Position in a ring of n slots: slot and phase parity of use number u, stepped as counters (u % n and u / n with a
-// run-time n and a 64-bit u are a division subroutine each, on the critical path of single-thread roles).
-struct RingPos {
-  int s;
-  uint32_t ph;
-  __device__ __forceinline__ void step(int n, int by = 1) { s += by; if (s >= n) { s -= n; ph ^= 1u; } }
-};
-
 __global__ void __launch_bounds__(DW1_THREADS, 1)
 mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
   const NumericArgs& a = g.na;
@@ -704,7 +851,7 @@ mlp_dw1_tc_kernel(const __grid_constant__ CUtensorMap tmD, MlpArgs g) {
             __threadfence();
             float tot = 0.f;
             for (int i2 = 0; i2 < per_r; ++i2) tot += __ldcg(mine + i2);
-            for (int i2 = 0; i2 < H / 32; ++i2) tot += __ldcg(sc.dist_head + (size_t)r * (H / 32) + i2);
+            for (int i2 = 0; i2 < H / MLP_HEAD_COLS; ++i2) tot += __ldcg(sc.dist_head + (size_t)r * (H / MLP_HEAD_COLS) + i2);
             a.dist2[(size_t)r * a.cap + j] = tot;
           }
         }
@@ -799,11 +946,11 @@ inline cudaError_t run_mlp_eval(NumericArgs& a, MlpScratch& s, MlpMaps& maps, co
   if (!mlp_make_maps(s, maps)) { *why = "mlp: could not encode the TMA tensor maps"; return cudaSuccess; }
   cudaError_t e;
   const TcLayout L = tc_forward_layout(s.H);
-  if ((e = cudaFuncSetAttribute(mlp_forward_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(mlp_risk_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total)) != cudaSuccess) return e;
   MlpArgs g{};
   g.na = a; g.sc = s; g.H = s.H; g.P = 0; g.j = 0;
   g.eval_blocks = (int)((s.n + 127) / 128); g.eval_slot = cur_slot; g.eval_parity = parity; g.eval_part = part;
-  mlp_forward_tc_kernel<true><<<a.R * g.eval_blocks, TC_THREADS, L.total, stream>>>(maps.tmW, g);
+  mlp_risk_tc_kernel<<<a.R * g.eval_blocks, TC_THREADS, L.total, stream>>>(maps.tmW, g);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   mlp_eval_finish_kernel<<<(a.R + 3) / 4, 128, 0, stream>>>(part, a.R, g.eval_blocks * 4, s.n, out);
   return cudaGetLastError();
@@ -816,8 +963,8 @@ inline cudaError_t run_mlp(NumericArgs& a, MlpScratch& s, MlpMaps& maps, int P, 
     *why = "mlp: could not encode the TMA tensor maps";
     return cudaSuccess;
   }
-  const TcLayout L = tc_forward_layout(s.H);
-  if ((e = cudaFuncSetAttribute(mlp_forward_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total)) != cudaSuccess) return e;
+  const TcFwdLayout L = tc_fwd_layout(s.H);
+  if ((e = cudaFuncSetAttribute(mlp_forward_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total)) != cudaSuccess) return e;
   const TcDw1Layout LD = tc_dw1_layout(s.H);
   if ((e = cudaFuncSetAttribute(mlp_dw1_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, LD.total)) != cudaSuccess) return e;
   int dev = 0, sms = 148;
@@ -827,12 +974,13 @@ inline cudaError_t run_mlp(NumericArgs& a, MlpScratch& s, MlpMaps& maps, int P, 
   const int dw1_grid = dw1_tiles < sms ? dw1_tiles : sms;      // one persistent CTA per SM
   MlpArgs g{};
   g.na = a; g.sc = s; g.H = s.H; g.P = P;
-  const int mtiles = s.m / 128;
+  const int fwd_tiles = a.R * s.Kmax * (s.m / 128) * (s.H > 256 ? 2 : 1);
+  const int fwd_grid = fwd_tiles < sms ? fwd_tiles : sms;
   for (long long u = 0; u < a.iters; ++u) {
     g.j = a.j0 + u;
     mlp_rows_kernel<<<a.R * s.Kmax, 128, 0, stream>>>(g);
-    mlp_forward_tc_kernel<false><<<a.R * s.Kmax * mtiles, TC_THREADS, L.total, stream>>>(maps.tmW, g);
-    mlp_head_kernel<<<a.R * (s.H / 32), MLP_HEAD_THREADS, 0, stream>>>(g);
+    mlp_forward_tc_kernel<<<fwd_grid, TC_THREADS, L.total, stream>>>(maps.tmW, g);
+    launch_mlp_head(g, stream);
     mlp_dw1_tc_kernel<<<dw1_grid, DW1_THREADS, LD.total, stream>>>(maps.tmD, g);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
