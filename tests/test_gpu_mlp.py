@@ -68,7 +68,9 @@ def run_mlp_case(B, data, w0, *, variant, P, K, m, eta, R, J, kind="exp", mu=1.0
 
 
 @pytest.mark.parametrize("variant", list(core.VARIANTS))
-@pytest.mark.parametrize("d,H,C,m,K,P", [(128, 64, 3, 128, 2, 4), (256, 192, 10, 256, 3, 5), (3072, 512, 10, 128, 4, 16)])
+@pytest.mark.parametrize("d,H,C,m,K,P", [(128, 64, 3, 128, 2, 4), (256, 192, 10, 256, 3, 5), (3072, 512, 10, 128, 4, 16),
+                                         # a hidden width whose halves are no multiple of 64, all 16 classes; 5..8 classes
+                                         (128, 320, 16, 128, 2, 4), (256, 128, 7, 128, 2, 3)])
 def test_mlp_variants_and_shapes(B, variant, d, H, C, m, K, P):
     data = inputs.make_mixture(4096, d, C, 0.5 if d < 1000 else 0.1, 95, "mlp2", H)
     w0 = inputs.mlp_init(d, H, C, 96)
