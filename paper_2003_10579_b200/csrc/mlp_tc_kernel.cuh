@@ -950,6 +950,7 @@ inline cudaError_t run_mlp_eval(NumericArgs& a, MlpScratch& s, MlpMaps& maps, co
   MlpArgs g{};
   g.na = a; g.sc = s; g.H = s.H; g.P = 0; g.j = 0;
   g.eval_blocks = (int)((s.n + 127) / 128); g.eval_slot = cur_slot; g.eval_parity = parity; g.eval_part = part;
+  if ((long long)a.R * g.eval_blocks > 0x7FFFFFFFll) { *why = "mlp: replicas x 128-row blocks of the data set exceed the grid limit 2^31 - 1"; return cudaSuccess; }
   mlp_risk_tc_kernel<<<a.R * g.eval_blocks, TC_THREADS, L.total, stream>>>(maps.tmW, g);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   mlp_eval_finish_kernel<<<(a.R + 3) / 4, 128, 0, stream>>>(part, a.R, g.eval_blocks * 4, s.n, out);
