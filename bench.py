@@ -121,6 +121,26 @@ def oracle_sample(wl, data, replica_ids, updates):
     return done, dt
 
 
+def oracle_workload(wl, data, variant, K, replica_ids, updates, t_interval=None):
+    """The CPU oracle on one thread on one (variant, K) run of a workload: `updates` updates of each given replica.
+    Returns the `cpu_oracle` object of a `workloads` entry."""
+    from threadpoolctl import threadpool_limits
+    from oracle.sim import OracleReplica
+    ti = wl.t_interval if t_interval is None else t_interval
+    w0 = wl.w0()
+    with threadpool_limits(limits=1):
+        t0 = time.perf_counter()
+        for r in replica_ids:
+            OracleReplica(model=data["model"], X=data["X"], y=data["y"], w0=w0, P=wl.P, K=K, variant=variant,
+                          delay_kind=wl.delay_kind, mu=wl.mu, shift=wl.shift, eta=wl.eta, m=wl.m, seed=wl.seed, replica=r,
+                          n_classes=wl.n_classes, hidden=wl.hidden, K0=wl.K0 if ti > 0 else 0, t_interval=ti).run(updates)
+        dt = time.perf_counter() - t0
+    n = len(replica_ids) * updates
+    return {"value": n / dt, "unit": "updates/s", "cores": 1, "kind": "oracle",
+            "sample": "%d replica(s) x %d updates of this run%s (%.1f s)" % (
+                len(replica_ids), updates, "" if ti == wl.t_interval else ", K doubling every %g time units" % ti, dt)}
+
+
 def _oracle_worker(index, reps, updates, ready, go, out):
     """One process of the all-cores baseline: makes its own copy of the data, waits for the common start,
     follows replicas [index*reps, (index+1)*reps) of every run."""
@@ -266,7 +286,7 @@ def timed_eval(sim, local, reps=3):
     return e0.elapsed_time(e1) / reps, sampler.finish()
 
 
-def run_other_workloads(inputs, peak, peaks, local, data2):
+def run_other_workloads(inputs, peak, peaks, local, data2, with_oracle=True):
     import torch
     out = []
     fp32_peak = 148 * 128 * 2 * 1.965e9 / 1e12       # TFLOP/s: 148 SMs x 128 FMA lanes x 2 flop at the 1965 MHz maximum clock
@@ -293,7 +313,8 @@ def run_other_workloads(inputs, peak, peaks, local, data2):
 
     # -- workload 1: small K-sync least squares; latency-bound by construction (1 MiB data set, 200 serial updates)
     wl = inputs.WORKLOADS[1]
-    dev = device_data(wl.make_data())
+    data = wl.make_data()
+    dev = device_data(data)
     for R in (65536, wl.replicas):       # the large launch first: the 64-replica run lasts 1.5 ms and would otherwise meet idle clocks
         sim = make_sim(wl, dev, "ksync", 2, R)
         ms, clocks = timed_run(sim, 3, wl.updates, wl.updates, local)
@@ -303,22 +324,28 @@ def run_other_workloads(inputs, peak, peaks, local, data2):
                               "read updates/s and us_per_update_step" if R == wl.replicas else
                               "same workload with 65536 replicas: the launch fills the GPU"))
         sim.close()
-    del dev
+    if with_oracle:      # the whole workload: all 64 replicas x 200 updates
+        out[-1]["cpu_oracle"] = oracle_workload(wl, data, "ksync", 2, range(wl.replicas), wl.updates)
+    del dev, data
 
     # -- workload 3: asynchronous variants with stale snapshots, logistic regression, K = 4
     wl = inputs.WORKLOADS[3]
-    dev = device_data(wl.make_data())
+    data = wl.make_data()
+    dev = device_data(data)
     for variant in ("kasync", "kbatchasync"):
         sim = make_sim(wl, dev, variant, 4, wl.replicas)
         ms, clocks = timed_run(sim, 3, 20, 200, local)
         out.append(entry(wl.name, wl, variant, 4, wl.replicas, 200, ms, clocks, last_K(sim, 200), peak))
         sim.close()
-    del dev
+        if with_oracle:
+            out[-1]["cpu_oracle"] = oracle_workload(wl, data, variant, 4, range(2), 100)
+    del dev, data
     torch.cuda.empty_cache()
 
     # -- workload 4: K-sync with K doubling 1 -> 8, softmax regression, the whole run (K depends on the clock)
     wl = inputs.WORKLOADS[4]
-    dev = device_data(wl.make_data())
+    data = wl.make_data()
+    dev = device_data(data)
     warm = make_sim(wl, dev, "ksync", 1, wl.replicas, interval=10.0)     # a short interval: the warm-up meets every K
     warm.run(20); warm.run(20); warm.run(20)
     warm.close()
@@ -333,18 +360,23 @@ def run_other_workloads(inputs, peak, peaks, local, data2):
     e["alu"] = {"bound": "alu", "achieved": tf, "peak": fp32_peak, "unit": "TFLOP/s", "frac": tf / fp32_peak}
     out.append(e)
     sim.close()
-    del dev
+    if with_oracle:      # a shorter interval for the timing run only, so that 300 updates meet K = 1, 2, 4 and 8
+        e["cpu_oracle"] = oracle_workload(wl, data, "ksync", 1, range(2), 300, t_interval=80.0)
+    del dev, data
     torch.cuda.empty_cache()
 
     # -- workload 5: K-batch-async MLP 3072-512-10 (bf16 tensor-core products over d)
     wl = inputs.WORKLOADS[5]
-    dev = device_data(wl.make_data())
+    data = wl.make_data()
+    dev = device_data(data)
     sim = make_sim(wl, dev, "kbatchasync", 4, wl.replicas)
     ms, clocks = timed_run(sim, 3, 10, 180, local)
     e = entry(wl.name, wl, "kbatchasync", 4, wl.replicas, 180, ms, clocks, last_K(sim, 180), peak,
               note="bytes counted for fp32 operands; the kernels read bf16 copies of X and W1, so DRAM traffic is lower")
     flops = 180 * wl.replicas * 4 * wl.m * (4 * wl.d * wl.hidden)      # forward and dW1 products, 2 flop per multiply-add
     e["tensor_tflops"] = flops / (ms * 1e-3) / 1e12
+    if with_oracle:
+        e["cpu_oracle"] = oracle_workload(wl, data, "kbatchasync", 4, range(1), 20)
     out.append(e)
     ms, clocks = timed_eval(sim, local, reps=2)
     tf = 2.0 * wl.n * wl.d * wl.hidden * wl.replicas / (ms * 1e-3) / 1e12
@@ -354,7 +386,7 @@ def run_other_workloads(inputs, peak, peaks, local, data2):
                 "roofline": {"bound": "tensor", "achieved": tf, "peak": tpeak, "unit": "TFLOP/s", "frac": tf / tpeak,
                              "note": "forward-only pass of the tcgen05 kernel over all 262144 rows for each of the 64 replicas"}})
     sim.close()
-    del dev
+    del dev, data
     torch.cuda.empty_cache()
 
     # -- the arrival process alone (clock-only mode, the runtime results of Section 3): replicas x updates per second
@@ -547,7 +579,7 @@ def main():
     torch.cuda.empty_cache()
 
     if world == 1 and not args.no_workloads:
-        line["workloads"] = run_other_workloads(inputs, peak, peaks, local, data)
+        line["workloads"] = run_other_workloads(inputs, peak, peaks, local, data, with_oracle=not args.no_cpu_baseline)
 
     if not args.no_e2e:
         # the public one-shot call on pinned host buffers: one step's work (all 32 runs, U updates from
