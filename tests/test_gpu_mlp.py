@@ -107,6 +107,27 @@ def test_mlp_growing_K_and_resume(B):
     a.close(); b.close()
 
 
+def test_mlp_results_do_not_depend_on_sharding(B):
+    """Replicas 3 and 4 of a six-replica handle and the same global replicas in a two-replica handle: every trace array
+    and every parameter bit for bit (the tile order of the persistent kernels depends on the replica count, the sums
+    must not)."""
+    data = inputs.make_mixture(2048, 256, 10, 0.5, 101, "mlp2", 512)
+    w0 = inputs.mlp_init(256, 512, 10, 102)
+    dev = to_device(data)
+    kw = dict(P=5, K=3, variant="kbatchasync", delay_kind="exp", mu=1.0, eta=0.02, m=128, seed=4)
+    full = B.Simulation(dev, n_replicas=6, **kw)
+    part = B.Simulation(dev, n_replicas=2, replica_base=3, **kw)
+    for s in (full, part):
+        s.set_params(torch.from_numpy(w0).cuda())
+        s.run(9)
+    tf, tp = full.trace(), part.trace()
+    for k in tf:
+        assert np.array_equal(tf[k][3:5], tp[k]), k
+    assert np.array_equal(full.params()[3:5], part.params())
+    assert np.array_equal(full.eval_loss()[3:5], part.eval_loss())
+    full.close(); part.close()
+
+
 def test_mlp_unsupported_shapes_are_refused(B):
     data = inputs.make_mixture(64, 128, 4, 0.5, 99, "mlp2", 100)
     with pytest.raises(B.SimError) as e:

@@ -46,6 +46,26 @@ def test_softmax_growing_K_scaled_fourth_workload(B):
     assert set(np.unique(tr["K"])) == {1, 2, 4, 8}
 
 
+@pytest.mark.parametrize("variant,C", [("ksync", 10), ("kasync", 10), ("kbatchasync", 13)])
+def test_softmax_results_do_not_depend_on_sharding(B, variant, C):
+    """Replicas 3 and 4 of a six-replica handle and the same global replicas in a two-replica handle, bit for bit
+    (both softmax kernels: up to 10 classes and 11 to 16)."""
+    import torch
+    from parity import to_device
+    data = inputs.make_mixture(1500, 3072 if C <= 10 else 1536, C, 0.05, 93)      # the 11..16-class kernel takes d <= 1536
+    dev = to_device(data)
+    kw = dict(P=4, K=2, variant=variant, delay_kind="exp", mu=1.0, eta=0.05, m=20, seed=6)
+    full = B.Simulation(dev, n_replicas=6, **kw)
+    part = B.Simulation(dev, n_replicas=2, replica_base=3, **kw)
+    for s in (full, part):
+        s.run(15)
+    tf, tp = full.trace(), part.trace()
+    for k in tf:
+        assert np.array_equal(tf[k][3:5], tp[k]), k
+    assert np.array_equal(full.params()[3:5], part.params())
+    full.close(); part.close()
+
+
 def test_softmax_unsupported_shapes_are_refused(B):
     data = inputs.make_mixture(64, 4096, 10, 0.5, 91)
     from parity import to_device
