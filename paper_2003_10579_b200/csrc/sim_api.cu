@@ -252,6 +252,10 @@ sim_status run_linear1(sim_handle* h, NumericArgs& a) {
   if (d4 <= 64) return launch_linear1<64, 1, 8>(h, a);
   if (d4 <= 128) return launch_linear1<128, 1, 4>(h, a);
   if (d4 <= 256) {
+    // many replicas (more than two CTAs per SM): one warp per replica with eight column chunks a thread.  Six such CTAs
+    // fit an SM (two 16 KB stages each) where five of 128 threads did, no block barrier is left in the tile loop, and the
+    // K-sweep workload runs 15 % faster; with few replicas the wider block is quicker per replica
+    if (!h->tune_rows && !h->tune_threads && a.R > 296) return launch_linear1<32, 8, 4>(h, a);
     const int rows = h->tune_rows ? h->tune_rows : 4;
     if (h->tune_threads == 256) return rows == 8 ? launch_linear1<256, 1, 8>(h, a) : launch_linear1<256, 1, 4>(h, a);
     return rows == 8 ? launch_linear1<128, 2, 8>(h, a) : rows == 2 ? launch_linear1<128, 2, 2>(h, a) : launch_linear1<128, 2, 4>(h, a);
