@@ -550,7 +550,7 @@ def main():
     ratio = measured_traffic_ratio()
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 # DRAM bytes of one step: dram read + write of an ncu capture of this kernel in the benchmark's launch
-                # shape (1024 replicas, five CTAs per SM) over its algorithmic bytes, times the step's algorithmic
+                # shape (1024 replicas, six one-warp CTAs per SM) over its algorithmic bytes, times the step's algorithmic
                 # bytes (traffic grows with the rows gathered); null if the committed summary does not state the ratio
                 "traffic": None if ratio is None else ratio * step_bytes,
                 "traffic_scaled_from": KSWEEP_PROFILE if ratio is not None else None,
