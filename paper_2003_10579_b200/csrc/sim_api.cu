@@ -226,8 +226,9 @@ sim_status launch_linear1(sim_handle* h, NumericArgs& a) {
   const size_t row_bytes = (size_t)d * 4;
   int S = h->tune_stages;
   if (S <= 0) {
-    // small rows: several CTAs per SM; long rows: one CTA per SM, or two when there are more replicas than SMs
-    const size_t budget = d <= 1024 ? (36u << 10) : (a.R > 148 ? (100u << 10) : (200u << 10));
+    // small rows: several CTAs per SM (with many replicas more CTAs of two stages beat fewer of three: rows of 2048 features
+    // 7.7 against 7.4 TB/s); long rows: one CTA per SM, or two when there are more replicas than SMs
+    const size_t budget = d <= 1024 ? (36u << 10) : (d <= 2048 && a.R > 296) ? (68u << 10) : (a.R > 148 ? (100u << 10) : (200u << 10));
     S = (int)(budget / ((size_t)T * row_bytes));
   }
   if (S < 2) S = 2;
@@ -250,17 +251,23 @@ sim_status run_linear1(sim_handle* h, NumericArgs& a) {
   // produces overlaps drawing indices and issuing copies with the arithmetic; with many, one warp per replica packs better
   if (d4 <= 32 && a.R > 296) return launch_linear1<32, 1, 8>(h, a);
   if (d4 <= 64) return launch_linear1<64, 1, 8>(h, a);
-  if (d4 <= 128) return launch_linear1<128, 1, 4>(h, a);
+  // With more than two replicas per SM narrow blocks with more column chunks a thread win (fewer warps meet at a tile's
+  // barrier - none in a one-warp block - and more blocks fit an SM).  Measured with eight simulations of 1024 replicas on
+  // concurrent streams, K = 8, m = 32: rows of 512 features 5.5 -> 7.1 TB/s, 1024 features 7.0 -> 8.1, 2048 features 6.2 -> 7.7.
+  const bool many = a.R > 296 && !h->tune_rows && !h->tune_threads;
+  if (d4 <= 128) {
+    if (many && linear1_smem_bytes(32, 8, 2, a.d, a.m) <= (size_t)(226 << 10)) return launch_linear1<32, 4, 8>(h, a);
+    return launch_linear1<128, 1, 4>(h, a);
+  }
   if (d4 <= 256) {
-    // many replicas (more than two CTAs per SM): one warp per replica with eight column chunks a thread.  Six such CTAs
-    // fit an SM (two 16 KB stages each) where five of 128 threads did, no block barrier is left in the tile loop, and the
-    // K-sweep workload runs 15 % faster; with few replicas the wider block is quicker per replica
-    if (!h->tune_rows && !h->tune_threads && a.R > 296) return launch_linear1<32, 8, 4>(h, a);
+    // one warp per replica with eight column chunks a thread: six such CTAs fit an SM (two 16 KB stages each) where five
+    // of 128 threads did, and the K-sweep workload runs 15 % faster; with few replicas the wider block is quicker per replica
+    if (many) return launch_linear1<32, 8, 4>(h, a);
     const int rows = h->tune_rows ? h->tune_rows : 4;
     if (h->tune_threads == 256) return rows == 8 ? launch_linear1<256, 1, 8>(h, a) : launch_linear1<256, 1, 4>(h, a);
     return rows == 8 ? launch_linear1<128, 2, 8>(h, a) : rows == 2 ? launch_linear1<128, 2, 2>(h, a) : launch_linear1<128, 2, 4>(h, a);
   }
-  if (d4 <= 512) return launch_linear1<256, 2, 4>(h, a);
+  if (d4 <= 512) return many ? launch_linear1<64, 8, 4>(h, a) : launch_linear1<256, 2, 4>(h, a);
   if (d4 <= 1024) {
     const int rows = h->tune_rows ? h->tune_rows : (a.R > 148 ? 2 : 4), threads = h->tune_threads ? h->tune_threads : 256;
     if (threads == 512 && d4 <= 1024) return rows == 2 ? launch_linear1<512, 2, 2>(h, a) : launch_linear1<512, 2, 4>(h, a);

@@ -83,11 +83,11 @@ def test_lsq_variants_and_shapes(B, variant, d, m, K, P):
 
 @pytest.mark.parametrize("variant", list(core.VARIANTS))
 @pytest.mark.parametrize("model,d,m", [("lsq", 1024, 32), ("lsq", 1000, 9), ("logistic", 516, 6), ("lsq", 64, 16),
-                                       ("logistic", 4096, 6), ("lsq", 2052, 5)])
+                                       ("logistic", 4096, 6), ("lsq", 2052, 5), ("lsq", 2048, 7), ("logistic", 300, 19)])
 def test_many_replicas_take_the_narrow_blocks(B, variant, model, d, m):
-    """With more than two replicas per SM rows of 513 to 1024 features go to blocks of one warp (eight column chunks a
-    thread) and rows of up to 128 features to blocks without the extra producer warp; with more than one per SM rows of
-    2049 to 4096 features go to four warps x eight chunks: same results, followed on four of 300 replicas."""
+    """With more than two replicas per SM the rows go to narrower blocks with more column chunks a thread (one warp for up
+    to 1024 features, two for up to 2048; rows of up to 128 features lose the extra producer warp); with more than one
+    per SM rows of 2049 to 4096 features go to four warps x eight chunks: same results, followed on four of 300 replicas."""
     data = inputs.make_lsq(3000, d, 0.1, 83) if model == "lsq" else inputs.make_logistic(3000, d, 0.05, 84)
     run_case(B, data, variant=variant, P=6, K=3, m=m, eta=0.02 if model == "lsq" else 0.01, R=300, J=30, kind="shifted_exp",
              mu=1.0, shift=0.5, base=2, replicas=[0, 1, 150, 299], chunks=[10], use_ref=model == "lsq")
