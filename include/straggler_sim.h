@@ -123,8 +123,10 @@ sim_status sim_set_adasync_loss(sim_handle* h, int32_t K0, double t_interval);
 /* Optional performance knobs of the linear-model kernels (0 = chosen from d): depth of the
  * shared-memory ring that stages sample rows ahead of the arithmetic (2..8), rows per tile (2 or
  * 4) and threads per replica (256 or 512) where the kernel for that d offers the choice.
- * Integer results never depend on them; fp32 results can differ in the last bits (summation
- * order). */
+ * Left at 0, the block shape also follows the number of replicas (narrow blocks with more columns
+ * a thread once there are more than two replicas per SM); setting tile_rows or threads switches
+ * that off.  Integer results never depend on any of this; fp32 results can differ in the last
+ * bits (summation order). */
 sim_status sim_set_tuning(sim_handle* h, int32_t stages, int32_t tile_rows, int32_t threads);
 
 /* Optional: make room for total_updates updates of trace now, so that later sim_run calls
