@@ -256,7 +256,7 @@ sim_status run_linear1(sim_handle* h, NumericArgs& a) {
   // up to 32 column chunks: with few replicas (at most two per SM the run is a chain of latencies) a second warp that only
   // produces overlaps drawing indices and issuing copies with the arithmetic; with many, one warp per replica packs better
   if (d4 <= 32 && a.R > 296) return launch_linear1<32, 1, 8>(h, a);
-  if (d4 <= 64) return launch_linear1<64, 1, 8>(h, a);
+  if (d4 <= 64) return (a.R > 296 && !h->tune_rows && !h->tune_threads) ? launch_linear1<32, 2, 8>(h, a) : launch_linear1<64, 1, 8>(h, a);
   // With more than two replicas per SM narrow blocks with more column chunks a thread win (fewer warps meet at a tile's
   // barrier - none in a one-warp block - and more blocks fit an SM).  Measured with eight simulations of 1024 replicas on
   // concurrent streams, K = 8, m = 32: rows of 512 features 5.5 -> 7.1 TB/s, 1024 features 7.0 -> 8.1, 2048 features 6.2 -> 7.7.

@@ -83,7 +83,7 @@ def test_lsq_variants_and_shapes(B, variant, d, m, K, P):
 
 @pytest.mark.parametrize("variant", list(core.VARIANTS))
 @pytest.mark.parametrize("model,d,m", [("lsq", 1024, 32), ("lsq", 1000, 9), ("logistic", 516, 6), ("lsq", 64, 16),
-                                       ("logistic", 4096, 6), ("lsq", 2052, 5), ("lsq", 2048, 7), ("logistic", 300, 19)])
+                                       ("logistic", 4096, 6), ("lsq", 2052, 5), ("lsq", 2048, 7), ("logistic", 300, 19), ("lsq", 256, 12)])
 def test_many_replicas_take_the_narrow_blocks(B, variant, model, d, m):
     """With more than two replicas per SM the rows go to narrower blocks with more column chunks a thread (one warp for up
     to 1024 features, two for up to 2048; rows of up to 128 features lose the extra producer warp); with more than one
