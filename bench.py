@@ -590,6 +590,9 @@ def main():
         kw = dict(P=wl.P, delay_kind=wl.delay_kind, mu=wl.mu, shift=wl.shift, eta=wl.eta, m=wl.m, seed=wl.seed,
                   n_replicas=R, replica_base=rank * R, iters=U, want=("t", "loss"))
         e2e_steps = max(1, min(args.steps, 10))
+        shape = (len(wl.runs), R, U)         # the traces land in pinned memory too
+        kw["out"] = {"t": torch.empty(shape, dtype=torch.float64).pin_memory().numpy(),
+                     "loss": torch.empty(shape, dtype=torch.float32).pin_memory().numpy()}
         sweep_host(host, wl.runs, **kw)
         barrier()
         t0 = time.perf_counter()

@@ -336,9 +336,11 @@ def simulate_host(data, *, P, K, variant, delay_kind, mu, shift=0.0, eta, m, see
 
 
 def sweep_host(data, runs, *, P, delay_kind, mu, shift=0.0, eta, m, seed, n_replicas, iters, replica_base=0, w0=None,
-               w_ref=None, want=("t", "loss")):
+               w_ref=None, want=("t", "loss"), out=None):
     """All (variant, K) pairs of `runs` on one HOST data set in one call: the data is copied in once,
-    the runs overlap on the device, the traces come back as [n_runs, R, iters] numpy arrays."""
+    the runs overlap on the device, the traces come back as [n_runs, R, iters] numpy arrays.  `out` may hold
+    arrays to write into (for instance views of pinned memory): C-contiguous, of that shape, float64 for "t" and
+    float32 for "loss" and "dist2"; missing ones are made here."""
     model = data["model"]
     prob = SimProblem(MODELS[model], 0, 0, 0, 0, None, None, None, None)
     keep = []
@@ -361,7 +363,15 @@ def sweep_host(data, runs, *, P, delay_kind, mu, shift=0.0, eta, m, seed, n_repl
     variants = np.array([VARIANTS[v] for v, _ in runs], np.int32)
     Ks = np.array([k for _, k in runs], np.int32)
     shape = (len(runs), n_replicas, iters)
-    out = {k: np.empty(shape, {"t": np.float64, "loss": np.float32, "dist2": np.float32}[k]) for k in want}
+    dtypes = {"t": np.float64, "loss": np.float32, "dist2": np.float32}
+    given, out = out or {}, {}
+    for k in want:
+        a = given.get(k)
+        if a is None:
+            a = np.empty(shape, dtypes[k])
+        elif a.shape != shape or a.dtype != dtypes[k] or not a.flags["C_CONTIGUOUS"] or not a.flags["WRITEABLE"]:
+            raise ValueError("out[%r] must be a writeable C-contiguous %s array of shape %r" % (k, np.dtype(dtypes[k]).name, shape))
+        out[k] = a
     ptrs = [C.c_void_p(out[k].ctypes.data) if k in out else None for k in ("t", "loss", "dist2")]
     _check(lib.sim_sweep_host(C.byref(prob), P, len(runs), C.c_void_p(variants.ctypes.data), C.c_void_p(Ks.ctypes.data),
                               SimDelay(DELAYS[delay_kind], mu, shift), eta, m, seed, n_replicas, replica_base,

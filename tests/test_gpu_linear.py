@@ -178,3 +178,9 @@ def test_sweep_on_host_buffers_matches_single_runs(B):
         sim.close()
         for k in ("t", "loss", "dist2"):
             assert np.array_equal(out[k][i], tr[k]), (variant, K, k)
+    # the same call writing into arrays of the caller (pinned memory here), and a wrong one refused before any work
+    mine = {"loss": torch.empty((len(runs), 6, 30), dtype=torch.float32).pin_memory().numpy()}
+    again = B.sweep_host(data, runs, iters=30, w_ref=data["w_star"], want=("t", "loss"), out=mine, **kw)
+    assert again["loss"] is mine["loss"] and np.array_equal(mine["loss"], out["loss"]) and np.array_equal(again["t"], out["t"])
+    with pytest.raises(ValueError):
+        B.sweep_host(data, runs, iters=30, want=("loss",), out={"loss": np.empty((len(runs), 6, 29), np.float32)}, **kw)
